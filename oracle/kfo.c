@@ -1,0 +1,192 @@
+/*
+ * kfo -- plain fp64 CPU oracle for the fused linear + epilogue + row-norm operator.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, obviously-correct definition that the
+ * CUDA library is checked against.  It shares no code, header, table or constant with the
+ * CUDA path; only tests, the smoke check and the bench's cpu_baseline / reference legs may
+ * build or call it.  Nothing here is tuned for speed: one accumulator per dot product,
+ * ascending k, libm for erf / tanh / exp, two-pass row statistics.  OpenMP only spreads
+ * independent rows over host cores; it changes no arithmetic.
+ *
+ * What is computed (the paper treats the framework reference of each task as the definition
+ * of the operator and demands an identical result -- Appendix E.1, "kernel generation prompt";
+ * the task families are Matmul+GELU+Softmax, Matmul+Swish+Scaling(+ResidualAdd), layernorm
+ * forward -- Tables 5-9; fused single-pass and online-normalisation forms are the expected
+ * kernel structure -- Section 3.2, algorithmic-structure descriptor).  For row i, column n:
+ *
+ *   acc = sum_{k=0}^{K-1} X[i,k] * W[n,k]                  (double, ascending k)
+ *   z   = acc + bias[n]                                     (if bias)
+ *   a   = act(z)     NONE: z
+ *                    GELU_ERF : 0.5 z (1 + erf(z / sqrt 2))
+ *                    GELU_TANH: 0.5 z (1 + tanh(sqrt(2/pi) (z + 0.044715 z^3)))
+ *                    SILU     : z / (1 + exp(-z))
+ *                    RELU     : max(z, 0)
+ *                    SIGMOID  : 1 / (1 + exp(-z))
+ *   a   = (double)scale * a
+ *   a   = a + R[i,n]                                        (if residual)
+ *   row op over n = 0..N-1:
+ *     NONE      y = a
+ *     SOFTMAX   m = max_n a ; y = exp(a - m) / sum_n exp(a - m)
+ *     LAYERNORM mu = (1/N) sum a ; v = (1/N) sum (a - mu)^2  (two passes, biased)
+ *               y = (a - mu) / sqrt(v + (double)eps) * gamma[n] + beta[n]
+ *     RMSNORM   y = a / sqrt((1/N) sum a^2 + (double)eps) * gamma[n]
+ *
+ * Inputs are the same bit patterns the GPU receives (fp32, or bf16 as uint16), widened
+ * exactly to double.  Outputs stay double.  Parity status: every function below is pinned by
+ * tests/test_oracle_pins.py (closed forms, brute force, invariants, library special cases).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+enum { KFO_F32 = 0, KFO_BF16 = 1, KFO_F64 = 2 };
+enum { KFO_ACT_NONE = 0, KFO_ACT_GELU_ERF = 1, KFO_ACT_GELU_TANH = 2, KFO_ACT_SILU = 3,
+       KFO_ACT_RELU = 4, KFO_ACT_SIGMOID = 5 };
+enum { KFO_NORM_NONE = 0, KFO_NORM_SOFTMAX = 1, KFO_NORM_LAYERNORM = 2, KFO_NORM_RMSNORM = 3 };
+
+/* exact widening of one stored element to double */
+static double widen(const void *p, long idx, int dtype)
+{
+    if (dtype == KFO_F32) {
+        return (double)((const float *)p)[idx];
+    } else if (dtype == KFO_BF16) {
+        uint32_t bits = ((uint32_t)((const uint16_t *)p)[idx]) << 16;
+        float f;
+        memcpy(&f, &bits, sizeof f);
+        return (double)f;
+    }
+    return ((const double *)p)[idx];
+}
+
+double kfo_act(int act, double z)
+{
+    switch (act) {
+    case KFO_ACT_NONE:      return z;
+    case KFO_ACT_GELU_ERF:  return 0.5 * z * (1.0 + erf(z / sqrt(2.0)));
+    case KFO_ACT_GELU_TANH: return 0.5 * z * (1.0 + tanh(sqrt(2.0 / M_PI) * (z + 0.044715 * z * z * z)));
+    case KFO_ACT_SILU:      return z / (1.0 + exp(-z));
+    case KFO_ACT_RELU:      return z > 0.0 ? z : 0.0;
+    case KFO_ACT_SIGMOID:   return 1.0 / (1.0 + exp(-z));
+    default:                return NAN;
+    }
+}
+
+/* row op on one row of doubles; a and y may alias */
+static void row_softmax(const double *a, double *y, long N)
+{
+    double m = a[0];
+    for (long n = 1; n < N; ++n) if (a[n] > m) m = a[n];
+    double s = 0.0;
+    for (long n = 0; n < N; ++n) s += exp(a[n] - m);
+    for (long n = 0; n < N; ++n) y[n] = exp(a[n] - m) / s;
+}
+
+static void row_layernorm(const double *a, double *y, long N, const void *gamma, const void *beta,
+                          double eps, int dtype)
+{
+    double mu = 0.0;
+    for (long n = 0; n < N; ++n) mu += a[n];
+    mu /= (double)N;
+    double v = 0.0;
+    for (long n = 0; n < N; ++n) v += (a[n] - mu) * (a[n] - mu);
+    v /= (double)N;
+    double sd = sqrt(v + eps);
+    for (long n = 0; n < N; ++n) {
+        double g = gamma ? widen(gamma, n, dtype) : 1.0;
+        double b = beta ? widen(beta, n, dtype) : 0.0;
+        y[n] = (a[n] - mu) / sd * g + b;
+    }
+}
+
+static void row_rmsnorm(const double *a, double *y, long N, const void *gamma, double eps, int dtype)
+{
+    double ms = 0.0;
+    for (long n = 0; n < N; ++n) ms += a[n] * a[n];
+    ms /= (double)N;
+    double r = sqrt(ms + eps);
+    for (long n = 0; n < N; ++n) {
+        double g = gamma ? widen(gamma, n, dtype) : 1.0;
+        y[n] = a[n] / r * g;
+    }
+}
+
+static void row_op(int norm, double *row, long N, const void *gamma, const void *beta, double eps,
+                   int dtype)
+{
+    if (N <= 0) return;
+    if (norm == KFO_NORM_SOFTMAX) row_softmax(row, row, N);
+    else if (norm == KFO_NORM_LAYERNORM) row_layernorm(row, row, N, gamma, beta, eps, dtype);
+    else if (norm == KFO_NORM_RMSNORM) row_rmsnorm(row, row, N, gamma, eps, dtype);
+}
+
+/*
+ * Fused operator: linear, element-wise epilogue, then the row op, literally composed.
+ * X [M,K] pitch ldx, W [N,K] pitch ldw, R [M,N] pitch ldr, Y [M,N] pitch ldy (elements);
+ * bias, gamma, beta [N]; all inputs share `dtype`.  Returns 0, or -1 on a bad enum.
+ */
+int kfo_linear_epilogue_rownorm(const void *X, long ldx, const void *W, long ldw, const void *bias,
+                                int act, float scale, const void *R, long ldr, int norm,
+                                const void *gamma, const void *beta, float eps, double *Y, long ldy,
+                                long M, long N, long K, int dtype)
+{
+    if (act < 0 || act > KFO_ACT_SIGMOID || norm < 0 || norm > KFO_NORM_RMSNORM) return -1;
+    if (dtype != KFO_F32 && dtype != KFO_BF16 && dtype != KFO_F64) return -1;
+    long i;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (i = 0; i < M; ++i) {
+        double *row = Y + i * ldy;
+        for (long n = 0; n < N; ++n) {
+            double acc = 0.0;
+            for (long k = 0; k < K; ++k)
+                acc += widen(X, i * ldx + k, dtype) * widen(W, n * ldw + k, dtype);
+            double z = acc;
+            if (bias) z += widen(bias, n, dtype);
+            double a = kfo_act(act, z);
+            a = (double)scale * a;
+            if (R) a += widen(R, i * ldr + n, dtype);
+            row[n] = a;
+        }
+        row_op(norm, row, N, gamma, beta, (double)eps, dtype);
+    }
+    return 0;
+}
+
+/* Stand-alone row ops: the last step above applied to a given [M,N]. */
+int kfo_row_norm(const void *X, long ldx, int norm, const void *gamma, const void *beta, float eps,
+                 double *Y, long ldy, long M, long N, int dtype)
+{
+    if (norm < 0 || norm > KFO_NORM_RMSNORM) return -1;
+    if (dtype != KFO_F32 && dtype != KFO_BF16 && dtype != KFO_F64) return -1;
+    long i;
+#pragma omp parallel for schedule(static)
+    for (i = 0; i < M; ++i) {
+        double *row = Y + i * ldy;
+        for (long n = 0; n < N; ++n) row[n] = widen(X, i * ldx + n, dtype);
+        row_op(norm, row, N, gamma, beta, (double)eps, dtype);
+    }
+    return 0;
+}
+
+int kfo_row_softmax(const void *X, long ldx, double *Y, long ldy, long M, long N, int dtype)
+{
+    return kfo_row_norm(X, ldx, KFO_NORM_SOFTMAX, NULL, NULL, 0.0f, Y, ldy, M, N, dtype);
+}
+
+int kfo_row_layernorm(const void *X, long ldx, const void *gamma, const void *beta, float eps,
+                      double *Y, long ldy, long M, long N, int dtype)
+{
+    return kfo_row_norm(X, ldx, KFO_NORM_LAYERNORM, gamma, beta, eps, Y, ldy, M, N, dtype);
+}
+
+int kfo_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}

@@ -1,0 +1,22 @@
+"""B200-native fused linear + epilogue + row-norm kernels behind a C-ABI library.
+
+``paper_2603_12440_b200.inputs`` (seeded synthetic inputs) imports without the CUDA library;
+everything else is the thin binding in ``paper_2603_12440_b200.binding`` and is loaded on first
+attribute access, so that it fails loudly, and only then, when ``libkf.so`` has not been built.
+"""
+from __future__ import annotations
+
+import importlib
+
+_BINDING_NAMES = (
+    "linear_epilogue", "linear_epilogue_rownorm", "row_softmax", "row_layernorm", "row_rmsnorm",
+    "workspace_bytes", "check_device_status", "status_string", "lib", "KfError",
+    "linear_epilogue_rownorm_host", "host_call_bytes", "tile_config", "library_path",
+)
+
+
+def __getattr__(name):
+    if name in _BINDING_NAMES or name == "binding":
+        mod = importlib.import_module(".binding", __name__)
+        return mod if name == "binding" else getattr(mod, name)
+    raise AttributeError(f"module {__name__!r} has no attribute {name!r}")
