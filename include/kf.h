@@ -1,0 +1,177 @@
+/*
+ * kf.h -- C ABI of the B200 (sm_100a) fused linear + epilogue + row-norm library.
+ *
+ * The paper frames an optimised kernel as a drop-in `forward` that must produce exactly the
+ * output of the framework reference operator, run in full on every call, and take its stream
+ * from the framework (Appendix E.1, main prompt: the result has to agree with the reference
+ * operator and nothing may be carried over from an earlier call; the Appendix E.2 listing takes
+ * the framework's current stream).  The operators are the task families it scores:
+ * Matmul+GELU+Softmax, Matmul+Swish+Scaling, Gemm+Sigmoid+Scaling+ResidualAdd (Appendix F.2,
+ * per-task comparison table), layernorm / rmsnorm / linear(+ReLU) forward (Appendix F.1,
+ * robust-kbench table), softmax and matmul with post-op (Section 4.4, oneDNN comparison table).
+ *
+ * Common conventions
+ *   - X is [M,K], W is [N,K] (so Y = X W^T), residual and Y are [M,N]; all row-major with the
+ *     last index contiguous.  ldx/ldw/ldr/ldy are row pitches in ELEMENTS.  bias/gamma/beta
+ *     are contiguous [N].
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller, unless the function name
+ *     ends in _host.  One dtype `dt` for all tensors of a call.  Accumulation and all epilogue
+ *     and row arithmetic are fp32; the result is rounded once (nearest-even) to `dt` at the
+ *     final store.  bf16 fused row-norm calls keep a bf16 intermediate of the pre-norm tile
+ *     (centred per tile for LayerNorm) before the final scaling; see kf_linear_epilogue_rownorm.
+ *   - Element-wise order: a = act(acc + bias[n]) * scale + residual[m,n].
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = the legacy
+ *     default stream), never synchronise, allocate no device memory and keep no result state.
+ *     Errors detectable on the host are returned at once and nothing is launched.
+ *   - `ws` is caller-owned device scratch of at least kf_workspace_bytes(...) bytes, 256-byte
+ *     aligned.  Its first 256 bytes hold a sticky device status word that kernels set only when
+ *     a bounded on-device wait gives up; zero it once with kf_workspace_init and read it with
+ *     kf_check_device_status.  Calls that share a `ws` must not overlap on the GPU.
+ *   - Alignment: fast paths need 16-byte aligned base pointers and row pitches; anything else
+ *     is served by slower generic kernels, never by the CPU.  There is no CPU fallback.
+ *   - M == 0 or N == 0: returns KF_OK and writes nothing.  K == 0: the accumulator is 0.
+ *   - Aliasing: Y may alias residual (same pitch) and, for the row functions, X.  Y must not
+ *     overlap X or W of the linear calls.  Inputs must be finite.
+ */
+#ifndef KF_H_
+#define KF_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    KF_OK = 0,
+    KF_ERR_INVALID_ARG = 1,   /* null pointer, negative size, pitch smaller than the row, bad enum */
+    KF_ERR_UNSUPPORTED = 2,   /* a combination no kernel serves */
+    KF_ERR_ALIGNMENT = 3,     /* pointer not aligned to its element size / workspace not 256-byte aligned */
+    KF_ERR_WORKSPACE = 4,     /* ws is NULL or smaller than kf_workspace_bytes */
+    KF_ERR_CUDA = 5,          /* a CUDA runtime / driver call failed (launch, tensor-map encode) */
+    KF_ERR_TIMEOUT = 6        /* device status word: a bounded wait inside a kernel gave up */
+} kf_status;
+
+typedef enum { KF_F32 = 0, KF_BF16 = 1 } kf_dtype;
+
+typedef enum {
+    KF_ACT_NONE = 0,
+    KF_ACT_GELU_ERF = 1,      /* 0.5 z (1 + erf(z / sqrt 2)) */
+    KF_ACT_GELU_TANH = 2,     /* 0.5 z (1 + tanh(sqrt(2/pi) (z + 0.044715 z^3))) */
+    KF_ACT_SILU = 3,          /* z / (1 + exp(-z))  ("Swish") */
+    KF_ACT_RELU = 4,
+    KF_ACT_SIGMOID = 5
+} kf_act;
+
+typedef enum {
+    KF_NORM_NONE = 0,
+    KF_NORM_SOFTMAX = 1,      /* exp(a - max) / sum exp(a - max) over the row */
+    KF_NORM_LAYERNORM = 2,    /* (a - mean) / sqrt(biased var + eps) * gamma + beta */
+    KF_NORM_RMSNORM = 3       /* a / sqrt(mean(a^2) + eps) * gamma */
+} kf_norm;
+
+/* Element-wise epilogue, fused so the data is passed over once (Section 3.2, level 1 of the
+ * algorithmic-structure descriptor). */
+typedef struct {
+    const void *bias;         /* [N] or NULL */
+    int32_t     act;          /* kf_act */
+    float       scale;        /* multiplies act(.); 1.0f = none */
+    const void *residual;     /* [M,N] or NULL */
+    int64_t     ldr;          /* residual row pitch in elements (ignored when residual is NULL) */
+} kf_epilogue;
+
+/* Row-wise reduction that follows the epilogue. */
+typedef struct {
+    int32_t     norm;         /* kf_norm */
+    const void *gamma;        /* [N] or NULL (= 1); LayerNorm and RMSNorm */
+    const void *beta;         /* [N] or NULL (= 0); LayerNorm only */
+    float       eps;          /* LayerNorm / RMSNorm */
+} kf_rownorm;
+
+/* Which kernel and tile shape a call resolves to (the hardware-aware table, Section 3.4:
+ * the best-measured instantiation of a templated kernel is the one that is used). */
+typedef struct {
+    int32_t kernel;           /* 0 none, 1 SIMT row-resident, 2 SIMT tiled, 3 tcgen05 */
+    int32_t bm, bn, bk;       /* CTA tile */
+    int32_t stages;           /* shared-memory pipeline depth */
+    int32_t cta_group;        /* 1 or 2 CTAs per MMA */
+    int32_t epilogue_warps;
+    int32_t row_scheme;       /* 0 none, 1 in-CTA rows, 2 split-N partials + normalise pass,
+                                 3 split-N partials + in-kernel deferred normalise, 4 un-fused */
+    int32_t grid;             /* CTAs launched by the main kernel */
+} kf_tile_config;
+
+/*
+ * Y = act(X W^T + bias) * scale + residual                                  (steps a1-a3, a5)
+ * ep may be NULL (no bias, no activation, scale 1, no residual).
+ */
+kf_status kf_linear_epilogue(const void *X, int64_t ldx, const void *W, int64_t ldw,
+                             void *Y, int64_t ldy, int64_t M, int64_t N, int64_t K, kf_dtype dt,
+                             const kf_epilogue *ep, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Y = rownorm(act(X W^T + bias) * scale + residual), the whole row of N outputs reduced inside
+ * the call (Section 3.2: level 2 of the algorithmic-structure descriptor, normalisation computed
+ * online while tiles stream by, and level 3 of the coordination descriptor, work-groups
+ * coordinating through global memory).  Row statistics are merged across N-tiles from per-tile
+ * partials: (max, sum exp) for softmax, (shift, sum, sum of squares) -> Chan's merge for
+ * LayerNorm, sum of squares for RMSNorm.  For bf16 with more than one N-tile the pre-norm tile
+ * is kept as bf16 between the two phases: exp(a - tile max) for softmax, a - tile shift for
+ * LayerNorm, a for RMSNorm.  rn->norm == KF_NORM_NONE makes this kf_linear_epilogue.
+ */
+kf_status kf_linear_epilogue_rownorm(const void *X, int64_t ldx, const void *W, int64_t ldw,
+                                     void *Y, int64_t ldy, int64_t M, int64_t N, int64_t K,
+                                     kf_dtype dt, const kf_epilogue *ep, const kf_rownorm *rn,
+                                     void *ws, size_t ws_bytes, void *stream);
+
+/* Stand-alone row operators on an existing [M,N] (step a6); Y may alias X. */
+kf_status kf_row_softmax(const void *X, int64_t ldx, void *Y, int64_t ldy, int64_t M, int64_t N,
+                         kf_dtype dt, void *stream);
+kf_status kf_row_layernorm(const void *X, int64_t ldx, const void *gamma, const void *beta,
+                           float eps, void *Y, int64_t ldy, int64_t M, int64_t N, kf_dtype dt,
+                           void *stream);
+kf_status kf_row_rmsnorm(const void *X, int64_t ldx, const void *gamma, float eps, void *Y,
+                         int64_t ldy, int64_t M, int64_t N, kf_dtype dt, void *stream);
+
+/*
+ * Host-buffer form of kf_linear_epilogue_rownorm: X, W, Y and the vectors / residual inside
+ * ep and rn are HOST pointers (pinned memory makes the copies asynchronous), tightly packed
+ * (pitch = row length).  `dev` is caller-owned device memory of at least
+ * kf_host_call_bytes(M,N,K,dt,has_residual,norm) bytes, 256-byte aligned; the call copies the
+ * inputs into it on `stream`, runs the device path there and copies Y back to the host.  The
+ * result is complete when `stream` has been synchronised by the caller.
+ */
+kf_status kf_linear_epilogue_rownorm_host(const void *X, const void *W, void *Y, int64_t M,
+                                          int64_t N, int64_t K, kf_dtype dt,
+                                          const kf_epilogue *ep, const kf_rownorm *rn, void *dev,
+                                          size_t dev_bytes, void *stream);
+size_t kf_host_call_bytes(int64_t M, int64_t N, int64_t K, kf_dtype dt, int has_residual,
+                          kf_norm norm);
+
+/* Bytes of `ws` the two linear calls need for this shape (always >= 256). */
+size_t kf_workspace_bytes(int64_t M, int64_t N, int64_t K, kf_dtype dt, kf_norm norm);
+
+/* Zero the status word (asynchronous on stream).  Call once after allocating ws. */
+kf_status kf_workspace_init(void *ws, size_t ws_bytes, void *stream);
+
+/* Synchronise `stream`, read the status word in ws, clear it, and return KF_OK or the recorded
+ * error.  *detail (may be NULL) receives a code naming the wait that gave up. */
+kf_status kf_check_device_status(void *ws, void *stream, uint32_t *detail);
+
+/* Step a7: resolve a call to its kernel and tile shape without launching anything.  `aligned`
+ * says whether all pointers and pitches of the call will be 16-byte aligned.  The environment
+ * variable KF_TILE_OVERRIDE="stages=S,epi=E,grid=G,scheme=R,kernel=Q" overrides table fields
+ * (for sweeps). */
+kf_status kf_tile_config_query(int64_t M, int64_t N, int64_t K, kf_dtype dt, kf_norm norm,
+                               int aligned, kf_tile_config *out);
+
+const char *kf_status_string(kf_status s);
+
+/* Library version as major * 10000 + minor * 100 + patch. */
+int kf_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KF_H_ */

@@ -9,10 +9,11 @@
  * independent rows over host cores; it changes no arithmetic.
  *
  * What is computed (the paper treats the framework reference of each task as the definition
- * of the operator and demands an identical result -- Appendix E.1, "kernel generation prompt";
- * the task families are Matmul+GELU+Softmax, Matmul+Swish+Scaling(+ResidualAdd), layernorm
- * forward -- Tables 5-9; fused single-pass and online-normalisation forms are the expected
- * kernel structure -- Section 3.2, algorithmic-structure descriptor).  For row i, column n:
+ * of the operator and demands an identical result -- Appendix E.1, main prompt; the task
+ * families are Matmul+GELU+Softmax, Matmul+Swish+Scaling(+ResidualAdd) -- Appendix F.2 per-task
+ * table -- and layernorm / rmsnorm forward -- Appendix F.1 robust-kbench table; fused
+ * single-pass and online-normalisation forms are the expected kernel structure -- Section 3.2,
+ * algorithmic-structure descriptor).  For row i, column n:
  *
  *   acc = sum_{k=0}^{K-1} X[i,k] * W[n,k]                  (double, ascending k)
  *   z   = acc + bias[n]                                     (if bias)

@@ -1,0 +1,287 @@
+"""Thin Python binding of the kf C-ABI library (``libkf.so``): argument marshalling only.
+
+torch supplies device memory and the current stream; every arithmetic step of the path runs in
+the library's CUDA kernels.  There is no CPU path: loading fails loudly when ``libkf.so`` has not
+been built (``python -m paper_2603_12440_b200.build``), and every call needs CUDA tensors.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+from typing import Optional
+
+import torch
+
+_PKG = Path(__file__).resolve().parent
+_LIB_PATH = _PKG / "libkf.so"
+
+KF_OK = 0
+DTYPE = {torch.float32: 0, torch.bfloat16: 1}
+ACT = {"none": 0, "gelu_erf": 1, "gelu_tanh": 2, "silu": 3, "relu": 4, "sigmoid": 5}
+NORM = {"none": 0, "softmax": 1, "layernorm": 2, "rmsnorm": 3}
+
+
+class KfError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} ({status})")
+
+
+class _Epilogue(ctypes.Structure):
+    _fields_ = [("bias", ctypes.c_void_p), ("act", ctypes.c_int32), ("scale", ctypes.c_float),
+                ("residual", ctypes.c_void_p), ("ldr", ctypes.c_int64)]
+
+
+class _RowNorm(ctypes.Structure):
+    _fields_ = [("norm", ctypes.c_int32), ("gamma", ctypes.c_void_p), ("beta", ctypes.c_void_p),
+                ("eps", ctypes.c_float)]
+
+
+class TileConfig(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("kernel", "bm", "bn", "bk", "stages", "cta_group", "epilogue_warps", "row_scheme", "grid")]
+
+    def as_dict(self):
+        return {n: getattr(self, n) for n, _ in self._fields_}
+
+
+_lib = None
+
+
+def library_path() -> Path:
+    return _LIB_PATH
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded C-ABI library.  Raises if it has not been built: there is no fallback."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not _LIB_PATH.exists():
+        raise ImportError(f"{_LIB_PATH} is missing: build it with `python -m paper_2603_12440_b200.build` "
+                          "(nvcc, sm_100a).  The kf operators have no CPU or eager fallback.")
+    L = ctypes.CDLL(str(_LIB_PATH))
+    vp, i64, sz, ci, cf = ctypes.c_void_p, ctypes.c_int64, ctypes.c_size_t, ctypes.c_int, ctypes.c_float
+    ep, rn = ctypes.POINTER(_Epilogue), ctypes.POINTER(_RowNorm)
+    L.kf_linear_epilogue.argtypes = [vp, i64, vp, i64, vp, i64, i64, i64, i64, ci, ep, vp, sz, vp]
+    L.kf_linear_epilogue_rownorm.argtypes = [vp, i64, vp, i64, vp, i64, i64, i64, i64, ci, ep, rn, vp, sz, vp]
+    L.kf_row_softmax.argtypes = [vp, i64, vp, i64, i64, i64, ci, vp]
+    L.kf_row_layernorm.argtypes = [vp, i64, vp, vp, cf, vp, i64, i64, i64, ci, vp]
+    L.kf_row_rmsnorm.argtypes = [vp, i64, vp, cf, vp, i64, i64, i64, ci, vp]
+    L.kf_linear_epilogue_rownorm_host.argtypes = [vp, vp, vp, i64, i64, i64, ci, ep, rn, vp, sz, vp]
+    L.kf_host_call_bytes.argtypes = [i64, i64, i64, ci, ci, ci]
+    L.kf_host_call_bytes.restype = sz
+    L.kf_workspace_bytes.argtypes = [i64, i64, i64, ci, ci]
+    L.kf_workspace_bytes.restype = sz
+    L.kf_workspace_init.argtypes = [vp, sz, vp]
+    L.kf_check_device_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
+    L.kf_tile_config_query.argtypes = [i64, i64, i64, ci, ci, ci, ctypes.POINTER(TileConfig)]
+    L.kf_status_string.argtypes = [ci]
+    L.kf_status_string.restype = ctypes.c_char_p
+    L.kf_version.argtypes = []
+    for name in ("kf_linear_epilogue", "kf_linear_epilogue_rownorm", "kf_row_softmax", "kf_row_layernorm",
+                 "kf_row_rmsnorm", "kf_linear_epilogue_rownorm_host", "kf_workspace_init",
+                 "kf_check_device_status", "kf_tile_config_query", "kf_version"):
+        getattr(L, name).restype = ci
+    _lib = L
+    return L
+
+
+def status_string(status: int) -> str:
+    return lib().kf_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str):
+    if status != KF_OK:
+        raise KfError(status, where)
+
+
+def _stream(stream) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return int(s.cuda_stream)
+
+
+def _mat(t: torch.Tensor, name: str):
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor: kf has no CPU path")
+    if t.dim() != 2 or (t.shape[1] > 1 and t.stride(1) != 1):
+        raise ValueError(f"{name} must be 2-D with a contiguous last dimension")
+    ld = t.stride(0) if t.shape[0] > 1 else max(t.shape[1], 1)
+    return t.data_ptr(), int(ld)
+
+
+def _vec(t: Optional[torch.Tensor], n: int, dtype, name: str) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda or t.dtype != dtype or t.dim() != 1 or t.shape[0] != n or (n > 1 and t.stride(0) != 1):
+        raise ValueError(f"{name} must be a contiguous CUDA vector of length {n} and the dtype of X")
+    return t.data_ptr()
+
+
+_ws_cache: dict = {}
+
+
+def workspace_bytes(M: int, N: int, K: int, dtype, norm: str = "none") -> int:
+    return int(lib().kf_workspace_bytes(M, N, K, DTYPE[dtype], NORM[norm]))
+
+
+def _workspace(device, nbytes: int, stream) -> torch.Tensor:
+    """Per-device scratch, grown on demand and status-initialised once per allocation."""
+    key = (device.index, _stream(stream))
+    ws = _ws_cache.get(key)
+    if ws is None or ws.numel() < nbytes:
+        ws = torch.empty(max(nbytes, 1 << 20), dtype=torch.uint8, device=device)
+        _check(lib().kf_workspace_init(ws.data_ptr(), ws.numel(), _stream(stream)), "kf_workspace_init")
+        _ws_cache[key] = ws
+    return ws
+
+
+def check_device_status(ws: Optional[torch.Tensor] = None, stream=None):
+    """Synchronise the stream and raise if a kernel recorded a device-side failure in ``ws``
+    (default: the binding's cached workspace of the current device and stream)."""
+    if ws is None:
+        ws = _ws_cache.get((torch.cuda.current_device(), _stream(stream)))
+        if ws is None:
+            torch.cuda.current_stream().synchronize()
+            return
+    detail = ctypes.c_uint32(0)
+    st = lib().kf_check_device_status(ws.data_ptr(), _stream(stream), ctypes.byref(detail))
+    if st != KF_OK:
+        raise KfError(st, f"device status (detail 0x{detail.value:x})")
+
+
+def tile_config(M: int, N: int, K: int, dtype, norm: str = "none", aligned: bool = True) -> dict:
+    """Kernel and tile shape a call of this shape resolves to (nothing is launched)."""
+    cfg = TileConfig()
+    _check(lib().kf_tile_config_query(M, N, K, DTYPE[dtype], NORM[norm], int(aligned), ctypes.byref(cfg)),
+           "kf_tile_config_query")
+    return cfg.as_dict()
+
+
+def linear_epilogue_rownorm(X, W, bias=None, act="none", scale=1.0, residual=None, norm="none", gamma=None,
+                            beta=None, eps=1e-5, out=None, ws=None, stream=None) -> torch.Tensor:
+    """rownorm(act(X @ W.T + bias) * scale + residual) through ``kf_linear_epilogue_rownorm``."""
+    L = lib()
+    if X.dtype not in DTYPE or W.dtype != X.dtype:
+        raise ValueError("X and W must both be float32 or both bfloat16")
+    M, K = X.shape
+    N, K2 = W.shape
+    if K2 != K:
+        raise ValueError("X is [M,K] and W is [N,K]")
+    px, ldx = _mat(X, "X")
+    pw, ldw = _mat(W, "W")
+    if out is None:
+        out = torch.empty((M, N), dtype=X.dtype, device=X.device)
+    elif out.dtype != X.dtype or tuple(out.shape) != (M, N):
+        raise ValueError("out must be [M,N] of the dtype of X")
+    py, ldy = _mat(out, "out")
+    ep = _Epilogue(_vec(bias, N, X.dtype, "bias"), ACT[act], float(scale), None, 0)
+    if residual is not None:
+        if residual.dtype != X.dtype or tuple(residual.shape) != (M, N):
+            raise ValueError("residual must be [M,N] of the dtype of X")
+        pr, ldr = _mat(residual, "residual")
+        ep.residual, ep.ldr = pr, ldr
+    rn = _RowNorm(NORM[norm], _vec(gamma, N, X.dtype, "gamma"), _vec(beta, N, X.dtype, "beta"), float(eps))
+    if ws is None:
+        ws = _workspace(X.device, int(L.kf_workspace_bytes(M, N, K, DTYPE[X.dtype], NORM[norm])), stream)
+    st = L.kf_linear_epilogue_rownorm(px, ldx, pw, ldw, py, ldy, M, N, K, DTYPE[X.dtype], ctypes.byref(ep),
+                                      ctypes.byref(rn), ws.data_ptr(), ws.numel(), _stream(stream))
+    _check(st, "kf_linear_epilogue_rownorm")
+    return out
+
+
+def linear_epilogue(X, W, bias=None, act="none", scale=1.0, residual=None, out=None, ws=None,
+                    stream=None) -> torch.Tensor:
+    """act(X @ W.T + bias) * scale + residual through ``kf_linear_epilogue``."""
+    L = lib()
+    if X.dtype not in DTYPE or W.dtype != X.dtype:
+        raise ValueError("X and W must both be float32 or both bfloat16")
+    M, K = X.shape
+    N, K2 = W.shape
+    if K2 != K:
+        raise ValueError("X is [M,K] and W is [N,K]")
+    px, ldx = _mat(X, "X")
+    pw, ldw = _mat(W, "W")
+    if out is None:
+        out = torch.empty((M, N), dtype=X.dtype, device=X.device)
+    elif out.dtype != X.dtype or tuple(out.shape) != (M, N):
+        raise ValueError("out must be [M,N] of the dtype of X")
+    py, ldy = _mat(out, "out")
+    ep = _Epilogue(_vec(bias, N, X.dtype, "bias"), ACT[act], float(scale), None, 0)
+    if residual is not None:
+        if residual.dtype != X.dtype or tuple(residual.shape) != (M, N):
+            raise ValueError("residual must be [M,N] of the dtype of X")
+        pr, ldr = _mat(residual, "residual")
+        ep.residual, ep.ldr = pr, ldr
+    if ws is None:
+        ws = _workspace(X.device, int(L.kf_workspace_bytes(M, N, K, DTYPE[X.dtype], 0)), stream)
+    st = L.kf_linear_epilogue(px, ldx, pw, ldw, py, ldy, M, N, K, DTYPE[X.dtype], ctypes.byref(ep),
+                              ws.data_ptr(), ws.numel(), _stream(stream))
+    _check(st, "kf_linear_epilogue")
+    return out
+
+
+def _row_call(X, out):
+    if X.dtype not in DTYPE:
+        raise ValueError("X must be float32 or bfloat16")
+    px, ldx = _mat(X, "X")
+    if out is None:
+        out = torch.empty_like(X, memory_format=torch.contiguous_format)
+    elif out.dtype != X.dtype or out.shape != X.shape:
+        raise ValueError("out must match X")
+    py, ldy = _mat(out, "out")
+    return px, ldx, py, ldy, out
+
+
+def row_softmax(X, out=None, stream=None) -> torch.Tensor:
+    px, ldx, py, ldy, out = _row_call(X, out)
+    M, N = X.shape
+    _check(lib().kf_row_softmax(px, ldx, py, ldy, M, N, DTYPE[X.dtype], _stream(stream)), "kf_row_softmax")
+    return out
+
+
+def row_layernorm(X, gamma=None, beta=None, eps=1e-5, out=None, stream=None) -> torch.Tensor:
+    px, ldx, py, ldy, out = _row_call(X, out)
+    M, N = X.shape
+    st = lib().kf_row_layernorm(px, ldx, _vec(gamma, N, X.dtype, "gamma"), _vec(beta, N, X.dtype, "beta"),
+                                float(eps), py, ldy, M, N, DTYPE[X.dtype], _stream(stream))
+    _check(st, "kf_row_layernorm")
+    return out
+
+
+def row_rmsnorm(X, gamma=None, eps=1e-5, out=None, stream=None) -> torch.Tensor:
+    px, ldx, py, ldy, out = _row_call(X, out)
+    M, N = X.shape
+    st = lib().kf_row_rmsnorm(px, ldx, _vec(gamma, N, X.dtype, "gamma"), float(eps), py, ldy, M, N,
+                              DTYPE[X.dtype], _stream(stream))
+    _check(st, "kf_row_rmsnorm")
+    return out
+
+
+def host_call_bytes(M: int, N: int, K: int, dtype, has_residual: bool, norm: str = "none") -> int:
+    return int(lib().kf_host_call_bytes(M, N, K, DTYPE[dtype], int(has_residual), NORM[norm]))
+
+
+def _host(t: Optional[torch.Tensor], name: str) -> Optional[int]:
+    if t is None:
+        return None
+    if t.is_cuda or not t.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous host tensor")
+    return t.data_ptr()
+
+
+def linear_epilogue_rownorm_host(X, W, out, dev, bias=None, act="none", scale=1.0, residual=None, norm="none",
+                                 gamma=None, beta=None, eps=1e-5, stream=None) -> torch.Tensor:
+    """Host-buffer form: X, W, vectors, residual and ``out`` are (pinned) host tensors, ``dev`` is a CUDA
+    uint8 arena of at least ``host_call_bytes`` bytes.  Copies in, runs the device path, copies Y back;
+    the result is valid after the stream has been synchronised."""
+    L = lib()
+    M, K = X.shape
+    N = W.shape[0]
+    ep = _Epilogue(_host(bias, "bias"), ACT[act], float(scale), _host(residual, "residual"), N)
+    rn = _RowNorm(NORM[norm], _host(gamma, "gamma"), _host(beta, "beta"), float(eps))
+    st = L.kf_linear_epilogue_rownorm_host(_host(X, "X"), _host(W, "W"), _host(out, "out"), M, N, K,
+                                           DTYPE[X.dtype], ctypes.byref(ep), ctypes.byref(rn), dev.data_ptr(),
+                                           dev.numel(), _stream(stream))
+    _check(st, "kf_linear_epilogue_rownorm_host")
+    return out

@@ -1,0 +1,283 @@
+// C ABI of the library: argument validation, the tile-shape table (step a7), workspace carve-up
+// and dispatch to the kernel files.  No torch types, no device allocation, no synchronisation
+// except in kf_check_device_status.
+#include <cstdlib>
+#include <cstring>
+
+#include "kf_tc.cuh"
+
+using namespace kf;
+
+namespace {
+
+inline size_t esize(int dt) { return dt == KF_F32 ? 4 : 2; }
+inline bool is_aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+inline size_t round256(size_t b) { return (b + 255) & ~(size_t)255; }
+
+struct Override {
+    int kernel = 0, grid = 0;
+};
+const Override& env_override() {
+    static Override o = [] {
+        Override v;
+        const char* e = std::getenv("KF_TILE_OVERRIDE");
+        if (!e) return v;
+        const char* p;
+        if ((p = std::strstr(e, "kernel="))) v.kernel = std::atoi(p + 7);
+        if ((p = std::strstr(e, "grid="))) v.grid = std::atoi(p + 5);
+        return v;
+    }();
+    return o;
+}
+
+// The table.  Shape classes and their winners; tensor-core rows carry the tile the kernel was
+// built with.  kernel: 1 SIMT row-resident, 2 SIMT tiled, 3 tcgen05.
+kf_status resolve(long long M, long long N, long long K, int dt, int norm, bool aligned, kf_tile_config* c) {
+    std::memset(c, 0, sizeof(*c));
+    if (M == 0 || N == 0) return KF_OK;
+    const Override& ov = env_override();
+    const bool tc_ok = dt == KF_BF16 && aligned && K > 0 && K % 8 == 0 && N % 8 == 0;
+    const double flops = 2.0 * (double)M * (double)N * (double)K;
+    bool use_tc = tc_ok && (flops >= 16.0e6 || (norm != KF_NORM_NONE && !simt_row_resident_ok(N)));
+    if (ov.kernel == 3 && tc_ok) use_tc = true;
+    if ((ov.kernel == 1 || ov.kernel == 2) &&
+        (norm == KF_NORM_NONE || dt == KF_F32 || simt_row_resident_ok(N)))
+        use_tc = false;
+    if (use_tc) {
+        c->kernel = 3;
+        tc_tile_shape(&c->bm, &c->bn, &c->bk, &c->stages, &c->epilogue_warps);
+        c->cta_group = 1;
+        c->row_scheme = norm == KF_NORM_NONE ? 0 : 2;
+        c->grid = tc_default_grid(M, N);
+        if (ov.grid > 0 && ov.grid < c->grid) c->grid = ov.grid;
+        return KF_OK;
+    }
+    bool rows = simt_row_resident_ok(N) && (norm != KF_NORM_NONE ? (M < 4096 || dt == KF_BF16) : (M <= 1024));
+    if (ov.kernel == 1 && simt_row_resident_ok(N)) rows = true;
+    if (ov.kernel == 2 && (norm == KF_NORM_NONE || dt == KF_F32)) rows = false;
+    if (rows) {
+        c->kernel = 1;
+        c->bn = (int)N; c->bk = 32; c->stages = 1; c->cta_group = 1; c->epilogue_warps = 8;
+        c->bm = 0;                                  // rows per CTA are picked from M at launch (1..8)
+        c->row_scheme = norm == KF_NORM_NONE ? 0 : 1;
+        return KF_OK;
+    }
+    if (norm != KF_NORM_NONE && dt == KF_BF16) return KF_ERR_UNSUPPORTED;   // would round the pre-norm row to bf16
+    c->kernel = 2;
+    c->bm = 64; c->bn = 64; c->bk = 16; c->stages = 1; c->cta_group = 1; c->epilogue_warps = 8;
+    c->row_scheme = norm == KF_NORM_NONE ? 0 : 4;
+    c->grid = (int)(((M + 63) / 64) * ((N + 63) / 64));
+    return KF_OK;
+}
+
+kf_status check_common(long long M, long long N, long long K, int dt) {
+    if (dt != KF_F32 && dt != KF_BF16) return KF_ERR_INVALID_ARG;
+    if (M < 0 || N < 0 || K < 0) return KF_ERR_INVALID_ARG;
+    if (M >= (1ll << 31) || N >= (1ll << 31) || K >= (1ll << 31)) return KF_ERR_UNSUPPORTED;
+    return KF_OK;
+}
+
+kf_status linear_impl(const void* X, int64_t ldx, const void* W, int64_t ldw, void* Y, int64_t ldy, int64_t M,
+                      int64_t N, int64_t K, int dt, const kf_epilogue* epi, const kf_rownorm* rni, void* ws,
+                      size_t ws_bytes, void* stream) {
+    kf_status s = check_common(M, N, K, dt);
+    if (s != KF_OK) return s;
+    EpilogueParams ep{nullptr, nullptr, 0, KF_ACT_NONE, 1.0f};
+    if (epi) {
+        if (epi->act < KF_ACT_NONE || epi->act > KF_ACT_SIGMOID) return KF_ERR_INVALID_ARG;
+        ep.bias = epi->bias; ep.residual = epi->residual; ep.ldr = epi->residual ? epi->ldr : 0;
+        ep.act = epi->act; ep.scale = epi->scale;
+    }
+    RowNormParams rn{KF_NORM_NONE, nullptr, nullptr, 0.f};
+    if (rni) {
+        if (rni->norm < KF_NORM_NONE || rni->norm > KF_NORM_RMSNORM) return KF_ERR_INVALID_ARG;
+        rn.norm = rni->norm;
+        if (rn.norm == KF_NORM_LAYERNORM || rn.norm == KF_NORM_RMSNORM) {
+            rn.gamma = rni->gamma; rn.eps = rni->eps;
+            if (rn.norm == KF_NORM_LAYERNORM) rn.beta = rni->beta;
+            if (!(rn.eps >= 0.f)) return KF_ERR_INVALID_ARG;
+        }
+    }
+    if (M == 0 || N == 0) return KF_OK;
+    if (!Y || (K > 0 && (!X || !W))) return KF_ERR_INVALID_ARG;
+    if (ldy < N || (K > 0 && (ldx < K || ldw < K)) || (ep.residual && ep.ldr < N)) return KF_ERR_INVALID_ARG;
+    const size_t es = esize(dt);
+    const void* ptrs[] = {X, W, Y, ep.bias, ep.residual, rn.gamma, rn.beta};
+    bool aligned = true;
+    for (const void* q : ptrs) {
+        if (q && !is_aligned(q, es)) return KF_ERR_ALIGNMENT;
+        if (q && !is_aligned(q, 16)) aligned = false;
+    }
+    if ((ldx * es) % 16 || (ldw * es) % 16 || (ldy * es) % 16 || (ep.residual && (ep.ldr * es) % 16)) aligned = false;
+    if (ws && !is_aligned(ws, 256)) return KF_ERR_ALIGNMENT;
+
+    kf_tile_config cfg;
+    s = resolve(M, N, K, dt, rn.norm, aligned, &cfg);
+    if (s != KF_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cfg.kernel == 3) {
+        const size_t need = kStatusBytes + (rn.norm != KF_NORM_NONE ? tc_partials_bytes(M, N) : 0);
+        if (!ws || ws_bytes < need) return KF_ERR_WORKSPACE;
+        return launch_tc_linear(X, ldx, W, ldw, Y, ldy, M, N, K, ep, rn, ws, env_override().grid, st, nullptr);
+    }
+    cudaError_t e = launch_simt_linear(X, ldx, W, ldw, Y, ldy, M, N, K, dt, ep, rn, cfg.kernel == 1, st, nullptr);
+    return e == cudaSuccess ? KF_OK : KF_ERR_CUDA;
+}
+
+kf_status row_impl(const void* X, int64_t ldx, void* Y, int64_t ldy, int64_t M, int64_t N, int dt,
+                   const RowNormParams& rn, void* stream) {
+    kf_status s = check_common(M, N, 0, dt);
+    if (s != KF_OK) return s;
+    if (!(rn.eps >= 0.f)) return KF_ERR_INVALID_ARG;
+    if (M == 0 || N == 0) return KF_OK;
+    if (!X || !Y || ldx < N || ldy < N) return KF_ERR_INVALID_ARG;
+    const size_t es = esize(dt);
+    const void* ptrs[] = {X, Y, rn.gamma, rn.beta};
+    for (const void* q : ptrs)
+        if (q && !is_aligned(q, es)) return KF_ERR_ALIGNMENT;
+    cudaError_t e = launch_row_norm(X, ldx, Y, ldy, M, N, dt, rn, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? KF_OK : KF_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+kf_status kf_linear_epilogue(const void* X, int64_t ldx, const void* W, int64_t ldw, void* Y, int64_t ldy,
+                             int64_t M, int64_t N, int64_t K, kf_dtype dt, const kf_epilogue* ep, void* ws,
+                             size_t ws_bytes, void* stream) {
+    return linear_impl(X, ldx, W, ldw, Y, ldy, M, N, K, (int)dt, ep, nullptr, ws, ws_bytes, stream);
+}
+
+kf_status kf_linear_epilogue_rownorm(const void* X, int64_t ldx, const void* W, int64_t ldw, void* Y, int64_t ldy,
+                                     int64_t M, int64_t N, int64_t K, kf_dtype dt, const kf_epilogue* ep,
+                                     const kf_rownorm* rn, void* ws, size_t ws_bytes, void* stream) {
+    return linear_impl(X, ldx, W, ldw, Y, ldy, M, N, K, (int)dt, ep, rn, ws, ws_bytes, stream);
+}
+
+kf_status kf_row_softmax(const void* X, int64_t ldx, void* Y, int64_t ldy, int64_t M, int64_t N, kf_dtype dt,
+                         void* stream) {
+    RowNormParams rn{KF_NORM_SOFTMAX, nullptr, nullptr, 0.f};
+    return row_impl(X, ldx, Y, ldy, M, N, (int)dt, rn, stream);
+}
+
+kf_status kf_row_layernorm(const void* X, int64_t ldx, const void* gamma, const void* beta, float eps, void* Y,
+                           int64_t ldy, int64_t M, int64_t N, kf_dtype dt, void* stream) {
+    RowNormParams rn{KF_NORM_LAYERNORM, gamma, beta, eps};
+    return row_impl(X, ldx, Y, ldy, M, N, (int)dt, rn, stream);
+}
+
+kf_status kf_row_rmsnorm(const void* X, int64_t ldx, const void* gamma, float eps, void* Y, int64_t ldy, int64_t M,
+                         int64_t N, kf_dtype dt, void* stream) {
+    RowNormParams rn{KF_NORM_RMSNORM, gamma, nullptr, eps};
+    return row_impl(X, ldx, Y, ldy, M, N, (int)dt, rn, stream);
+}
+
+size_t kf_workspace_bytes(int64_t M, int64_t N, int64_t K, kf_dtype dt, kf_norm norm) {
+    (void)K;
+    size_t b = kStatusBytes;
+    if (dt == KF_BF16 && norm != KF_NORM_NONE && M > 0 && N > 0) b += tc_partials_bytes(M, N);
+    return round256(b);
+}
+
+kf_status kf_workspace_init(void* ws, size_t ws_bytes, void* stream) {
+    if (!ws || ws_bytes < (size_t)kStatusBytes) return KF_ERR_WORKSPACE;
+    if (!is_aligned(ws, 256)) return KF_ERR_ALIGNMENT;
+    return cudaMemsetAsync(ws, 0, kStatusBytes, static_cast<cudaStream_t>(stream)) == cudaSuccess ? KF_OK
+                                                                                                   : KF_ERR_CUDA;
+}
+
+kf_status kf_check_device_status(void* ws, void* stream, uint32_t* detail) {
+    if (!ws) return KF_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaStreamSynchronize(st) != cudaSuccess) return KF_ERR_CUDA;
+    uint32_t h[2] = {0, 0};
+    if (cudaMemcpy(h, ws, sizeof(h), cudaMemcpyDeviceToHost) != cudaSuccess) return KF_ERR_CUDA;
+    if (detail) *detail = h[1];
+    if (h[0] == 0) return KF_OK;
+    if (cudaMemset(ws, 0, kStatusBytes) != cudaSuccess) return KF_ERR_CUDA;
+    return h[0] <= (uint32_t)KF_ERR_TIMEOUT ? (kf_status)h[0] : KF_ERR_CUDA;
+}
+
+size_t kf_host_call_bytes(int64_t M, int64_t N, int64_t K, kf_dtype dt, int has_residual, kf_norm norm) {
+    if (M < 0 || N < 0 || K < 0) return 0;
+    const size_t es = esize((int)dt);
+    size_t b = 0;
+    b += round256((size_t)M * K * es);                       // X
+    b += round256((size_t)N * K * es);                       // W
+    b += round256((size_t)M * N * es);                       // Y
+    if (has_residual) b += round256((size_t)M * N * es);     // residual
+    b += 3 * round256((size_t)N * es);                       // bias, gamma, beta
+    b += kf_workspace_bytes(M, N, K, dt, norm);
+    return b;
+}
+
+kf_status kf_linear_epilogue_rownorm_host(const void* X, const void* W, void* Y, int64_t M, int64_t N, int64_t K,
+                                          kf_dtype dt, const kf_epilogue* ep, const kf_rownorm* rn, void* dev,
+                                          size_t dev_bytes, void* stream) {
+    kf_status s = check_common(M, N, K, (int)dt);
+    if (s != KF_OK) return s;
+    if (M == 0 || N == 0) return KF_OK;
+    if (!Y || (K > 0 && (!X || !W))) return KF_ERR_INVALID_ARG;
+    const int norm = rn ? rn->norm : KF_NORM_NONE;
+    if (norm < KF_NORM_NONE || norm > KF_NORM_RMSNORM) return KF_ERR_INVALID_ARG;
+    const bool has_res = ep && ep->residual;
+    if (!dev || dev_bytes < kf_host_call_bytes(M, N, K, dt, has_res, (kf_norm)norm)) return KF_ERR_WORKSPACE;
+    if (!is_aligned(dev, 256)) return KF_ERR_ALIGNMENT;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t es = esize((int)dt);
+    uint8_t* cur = static_cast<uint8_t*>(dev);
+    bool copy_ok = true;
+    auto stage = [&](const void* host, size_t bytes) -> void* {
+        void* d = cur;
+        cur += round256(bytes);
+        if (host && bytes) copy_ok &= cudaMemcpyAsync(d, host, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+        return host ? d : nullptr;
+    };
+    void* dX = stage(K > 0 ? X : nullptr, (size_t)M * K * es);
+    void* dW = stage(K > 0 ? W : nullptr, (size_t)N * K * es);
+    void* dY = cur;
+    cur += round256((size_t)M * N * es);
+    kf_epilogue dep{nullptr, KF_ACT_NONE, 1.0f, nullptr, 0};
+    if (ep) dep = *ep;
+    if (has_res) { dep.residual = stage(ep->residual, (size_t)M * N * es); dep.ldr = N; }
+    dep.bias = stage(ep ? ep->bias : nullptr, (size_t)N * es);
+    kf_rownorm drn{KF_NORM_NONE, nullptr, nullptr, 0.f};
+    if (rn) drn = *rn;
+    drn.gamma = stage(rn ? rn->gamma : nullptr, (size_t)N * es);
+    drn.beta = stage(rn ? rn->beta : nullptr, (size_t)N * es);
+    void* ws = cur;
+    const size_t ws_bytes = kf_workspace_bytes(M, N, K, dt, (kf_norm)norm);
+    copy_ok &= cudaMemsetAsync(ws, 0, kStatusBytes, st) == cudaSuccess;
+    if (!copy_ok) return KF_ERR_CUDA;
+    s = linear_impl(dX, K, dW, K, dY, N, M, N, K, (int)dt, &dep, &drn, ws, ws_bytes, stream);
+    if (s != KF_OK) return s;
+    if (cudaMemcpyAsync(Y, dY, (size_t)M * N * es, cudaMemcpyDeviceToHost, st) != cudaSuccess) return KF_ERR_CUDA;
+    return KF_OK;
+}
+
+kf_status kf_tile_config_query(int64_t M, int64_t N, int64_t K, kf_dtype dt, kf_norm norm, int aligned,
+                               kf_tile_config* out) {
+    if (!out) return KF_ERR_INVALID_ARG;
+    kf_status s = check_common(M, N, K, (int)dt);
+    if (s != KF_OK) return s;
+    if (norm < KF_NORM_NONE || norm > KF_NORM_RMSNORM) return KF_ERR_INVALID_ARG;
+    return resolve(M, N, K, (int)dt, (int)norm, aligned != 0, out);
+}
+
+const char* kf_status_string(kf_status s) {
+    switch (s) {
+    case KF_OK: return "KF_OK";
+    case KF_ERR_INVALID_ARG: return "KF_ERR_INVALID_ARG";
+    case KF_ERR_UNSUPPORTED: return "KF_ERR_UNSUPPORTED";
+    case KF_ERR_ALIGNMENT: return "KF_ERR_ALIGNMENT";
+    case KF_ERR_WORKSPACE: return "KF_ERR_WORKSPACE";
+    case KF_ERR_CUDA: return "KF_ERR_CUDA";
+    case KF_ERR_TIMEOUT: return "KF_ERR_TIMEOUT";
+    default: return "KF_ERR_UNKNOWN";
+    }
+}
+
+int kf_version(void) { return 100; }
+
+}  // extern "C"

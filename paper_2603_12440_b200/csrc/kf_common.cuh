@@ -1,0 +1,142 @@
+// Shared device helpers for the kf kernels (sm_100a).  Internal: not part of the C ABI.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/kf.h"
+
+namespace kf {
+
+constexpr int kStatusBytes = 256;          // head of every workspace: [0] status, [1] detail
+
+// ---- element access -----------------------------------------------------------------------
+template <typename T> struct Elem;
+template <> struct Elem<float> {
+    static constexpr int kVec = 4;         // elements per 16-byte vector
+    __device__ __forceinline__ static float load(const float* p) { return *p; }
+    __device__ __forceinline__ static void store(float* p, float v) { *p = v; }
+};
+template <> struct Elem<__nv_bfloat16> {
+    static constexpr int kVec = 8;
+    __device__ __forceinline__ static float load(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+    __device__ __forceinline__ static void store(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+};
+
+__device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);      // .x = lo (low half), .y = hi
+    return *reinterpret_cast<uint32_t*>(&h);
+}
+
+// unpack one 16-byte vector into floats / pack back
+template <typename T> __device__ __forceinline__ void unpack(const uint4& v, float* f);
+template <> __device__ __forceinline__ void unpack<float>(const uint4& v, float* f) {
+    f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y);
+    f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+}
+template <> __device__ __forceinline__ void unpack<__nv_bfloat16>(const uint4& v, float* f) {
+    f[0] = bf16lo(v.x); f[1] = bf16hi(v.x); f[2] = bf16lo(v.y); f[3] = bf16hi(v.y);
+    f[4] = bf16lo(v.z); f[5] = bf16hi(v.z); f[6] = bf16lo(v.w); f[7] = bf16hi(v.w);
+}
+template <typename T> __device__ __forceinline__ uint4 pack(const float* f);
+template <> __device__ __forceinline__ uint4 pack<float>(const float* f) {
+    return make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]), __float_as_uint(f[3]));
+}
+template <> __device__ __forceinline__ uint4 pack<__nv_bfloat16>(const float* f) {
+    return make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
+}
+
+// ---- activations (fp32) --------------------------------------------------------------------
+// ACCURATE = true is used by the fp32 paths (1e-4 absolute gate on small outputs); the bf16
+// tensor-core epilogue uses the fast forms, whose error (< 1e-6 relative-to-|z|) is far below a
+// bf16 ulp.
+constexpr float kLog2e = 1.4426950408889634f;
+
+__device__ __forceinline__ float fast_exp(float x) { return exp2f(x * kLog2e); }   // ex2.approx
+
+__device__ __forceinline__ float fast_rcp(float x) {
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+
+// erf via Abramowitz-Stegun 7.1.26 (|err| <= 1.5e-7): two MUFU ops and a degree-5 Horner chain.
+__device__ __forceinline__ float fast_erf(float x) {
+    float ax = fabsf(x);
+    float t = fast_rcp(fmaf(0.3275911f, ax, 1.0f));
+    float p = fmaf(t, 1.061405429f, -1.453152027f);
+    p = fmaf(p, t, 1.421413741f);
+    p = fmaf(p, t, -0.284496736f);
+    p = fmaf(p, t, 0.254829592f);
+    p *= t;
+    float e = exp2f(-ax * ax * kLog2e);
+    float r = fmaf(-p, e, 1.0f);
+    return copysignf(r, x);
+}
+
+template <bool ACCURATE>
+__device__ __forceinline__ float apply_act(int act, float z) {
+    switch (act) {
+    case KF_ACT_GELU_ERF:
+        if (ACCURATE) return 0.5f * z * (1.0f + erff(z * 0.70710678118654752f));
+        return 0.5f * z * (1.0f + fast_erf(z * 0.70710678118654752f));
+    case KF_ACT_GELU_TANH: {
+        float u = 0.7978845608028654f * fmaf(0.044715f * z, z * z, z);
+        if (ACCURATE) return 0.5f * z * (1.0f + tanhf(u));
+        // tanh(u) = 1 - 2 / (exp(2u) + 1)
+        float e = exp2f(fminf(u * (2.0f * kLog2e), 80.0f));
+        return 0.5f * z * (2.0f - 2.0f * fast_rcp(e + 1.0f));
+    }
+    case KF_ACT_SILU:
+        if (ACCURATE) return z / (1.0f + expf(-z));
+        return z * fast_rcp(1.0f + exp2f(fminf(-z * kLog2e, 80.0f)));
+    case KF_ACT_RELU:
+        return fmaxf(z, 0.0f);
+    case KF_ACT_SIGMOID:
+        if (ACCURATE) return 1.0f / (1.0f + expf(-z));
+        return fast_rcp(1.0f + exp2f(fminf(-z * kLog2e, 80.0f)));
+    default:
+        return z;
+    }
+}
+
+// ---- warp / block reductions -----------------------------------------------------------------
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+    return v;
+}
+
+// ---- launch parameter blocks shared by the .cu files ---------------------------------------------
+struct EpilogueParams {
+    const void* bias;
+    const void* residual;
+    long long ldr;
+    int act;
+    float scale;
+};
+
+struct RowNormParams {
+    int norm;
+    const void* gamma;
+    const void* beta;
+    float eps;
+};
+
+// host-side launchers implemented in the kernel files; all return cudaError_t from the launch
+cudaError_t launch_row_norm(const void* X, long long ldx, void* Y, long long ldy, long long M, long long N,
+                            int dt, const RowNormParams& rn, cudaStream_t st);
+cudaError_t launch_simt_linear(const void* X, long long ldx, const void* W, long long ldw, void* Y,
+                               long long ldy, long long M, long long N, long long K, int dt,
+                               const EpilogueParams& ep, const RowNormParams& rn, bool row_resident,
+                               cudaStream_t st, int* grid_out);
+bool simt_row_resident_ok(long long N);
+
+}  // namespace kf

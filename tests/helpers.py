@@ -1,0 +1,67 @@
+"""Shared pieces of the GPU parity tests: moving seeded problems to the device, reading results
+back as float64, and the tolerance the build is held to.
+
+Tolerance (from the build's target statement): fp32 calls -- max abs error <= 1e-4 on the final
+output; bf16 calls (fp32 accumulate) -- abs error <= 2e-2 AND error <= 1e-2 * max(|ref|, s) for
+every element, s = RMS of the oracle tensor (the relative test is floored at tensor scale so that
+outputs crossing zero are judged sensibly).  fp32 calls are additionally held to a floored relative
+5e-5, because 1e-4 absolute is loose for softmax outputs of size 1/N.
+"""
+import numpy as np
+import torch
+
+from paper_2603_12440_b200 import inputs
+
+
+def to_device(a, dtype: str, device="cuda"):
+    """numpy float32 array, or uint16 bf16 bit patterns, -> CUDA tensor of that dtype."""
+    if a is None:
+        return None
+    if dtype == "bf16":
+        return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).view(torch.bfloat16).to(device)
+    return torch.from_numpy(np.ascontiguousarray(a)).to(device)
+
+
+def to_f64(t: torch.Tensor) -> np.ndarray:
+    """CUDA result -> float64 numpy, exactly."""
+    t = t.detach().cpu().contiguous()
+    if t.dtype == torch.bfloat16:
+        return inputs.to_f64(t.view(torch.int16).numpy().view(np.uint16))
+    return t.numpy().astype(np.float64)
+
+
+def error_report(got: np.ndarray, ref: np.ndarray) -> dict:
+    err = np.abs(got - ref)
+    s = float(np.sqrt(np.mean(ref * ref))) if ref.size else 0.0
+    denom = np.maximum(np.abs(ref), s) if s > 0 else np.ones_like(ref)
+    nu = err / (np.abs(ref) + 1e-12)
+    cos = float((got * ref).sum() / (np.linalg.norm(got) * np.linalg.norm(ref) + 1e-300)) if ref.size else 1.0
+    return {"max_abs": float(err.max()) if err.size else 0.0,
+            "max_rel_floored": float((err / denom).max()) if err.size else 0.0,
+            "rms_ref": s, "max_ref": float(np.abs(ref).max()) if ref.size else 0.0,
+            "frac_nu_lt_1e-2": float((nu < 1e-2).mean()) if ref.size else 1.0, "cosine": cos}
+
+
+def assert_parity(got: np.ndarray, ref: np.ndarray, dtype: str, what: str = ""):
+    assert got.shape == ref.shape, (what, got.shape, ref.shape)
+    assert np.all(np.isfinite(got)), f"{what}: non-finite output"
+    r = error_report(got, ref)
+    if dtype == "f32":
+        assert r["max_abs"] <= 1e-4, (what, r)
+        assert r["max_rel_floored"] <= 5e-5, (what, r)
+    else:
+        assert r["max_abs"] <= 2e-2, (what, r)
+        assert r["max_rel_floored"] <= 1e-2, (what, r)
+    return r
+
+
+def problem_to_device(p):
+    d = p.dtype
+    return {k: to_device(getattr(p, k), d) for k in ("X", "W", "bias", "residual", "gamma", "beta")}
+
+
+def oracle_of(p):
+    from oracle import kfo
+    if p.K == 0:
+        return kfo.row_norm(p.X, p.norm, p.gamma, p.beta, p.eps)
+    return kfo.linear_epilogue_rownorm(p.X, p.W, p.bias, p.act, p.scale, p.residual, p.norm, p.gamma, p.beta, p.eps)

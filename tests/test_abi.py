@@ -1,0 +1,118 @@
+"""CPU-side checks of the C-ABI library: it loads, exports every symbol the header declares, and its
+host logic (argument validation, workspace sizing, tile table) behaves.  No kernel is launched."""
+import ctypes
+import re
+from pathlib import Path
+
+import pytest
+
+ROOT = Path(__file__).resolve().parent.parent
+
+
+@pytest.fixture(scope="module")
+def kf():
+    from paper_2603_12440_b200 import build
+    build.build()
+    from paper_2603_12440_b200 import binding
+    binding.lib()
+    return binding
+
+
+def test_exports_every_declared_symbol(kf):
+    header = (ROOT / "include" / "kf.h").read_text()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(kf_[a-z_0-9]+)\s*\(", header))
+    assert {"kf_linear_epilogue", "kf_linear_epilogue_rownorm", "kf_row_softmax", "kf_row_layernorm"} <= declared
+    L = kf.lib()
+    for name in sorted(declared):
+        assert hasattr(L, name), f"libkf.so does not export {name}"
+
+
+def test_library_has_no_driver_link_dependency(kf):
+    # the library must load on a machine without libcuda (this test runs on such a machine)
+    assert kf.lib().kf_version() >= 100
+
+
+def test_status_strings(kf):
+    names = [kf.status_string(i) for i in range(7)]
+    assert names == ["KF_OK", "KF_ERR_INVALID_ARG", "KF_ERR_UNSUPPORTED", "KF_ERR_ALIGNMENT",
+                     "KF_ERR_WORKSPACE", "KF_ERR_CUDA", "KF_ERR_TIMEOUT"]
+    assert kf.status_string(99) == "KF_ERR_UNKNOWN"
+
+
+def test_workspace_bytes(kf):
+    import torch
+    assert kf.workspace_bytes(128, 256, 256, torch.float32, "softmax") == 256
+    assert kf.workspace_bytes(8192, 4096, 4096, torch.bfloat16, "none") == 256
+    # bf16 row-norm: one float4 per row per 256-column tile, rows padded to 128, after the status block
+    assert kf.workspace_bytes(4096, 8192, 2048, torch.bfloat16, "layernorm") == 256 + 32 * 32 * 128 * 16
+    assert kf.workspace_bytes(2048, 32768, 1024, torch.bfloat16, "softmax") == 256 + 16 * 128 * 128 * 16
+    assert kf.workspace_bytes(100, 300, 64, torch.bfloat16, "rmsnorm") == 256 + 1 * 2 * 128 * 16
+
+
+def test_tile_table_on_the_five_configs(kf):
+    import torch
+    c1 = kf.tile_config(128, 256, 256, torch.float32, "softmax")
+    assert c1["kernel"] == 1 and c1["row_scheme"] == 1            # fp32: CUDA cores, rows resident in a CTA
+    c3 = kf.tile_config(8192, 4096, 4096, torch.bfloat16, "none")
+    assert (c3["kernel"], c3["bm"], c3["bn"], c3["bk"], c3["row_scheme"]) == (3, 128, 256, 64, 0)
+    assert 1 <= c3["grid"] <= 1024
+    c4 = kf.tile_config(4096, 8192, 2048, torch.bfloat16, "layernorm")
+    assert c4["kernel"] == 3 and c4["row_scheme"] == 2
+    c5 = kf.tile_config(2048, 32768, 1024, torch.bfloat16, "softmax")
+    assert c5["kernel"] == 3 and c5["row_scheme"] == 2
+    # unaligned bf16 falls to the generic CUDA-core kernels; a long unaligned bf16 row-norm is refused
+    assert kf.tile_config(512, 512, 520, torch.bfloat16, "none", aligned=False)["kernel"] in (1, 2)
+    with pytest.raises(kf.KfError) as e:
+        kf.tile_config(512, 4104, 520, torch.bfloat16, "softmax", aligned=False)
+    assert e.value.status == 2
+    # fp32 never goes to the tensor cores
+    assert kf.tile_config(8192, 8192, 8192, torch.float32, "none")["kernel"] == 2
+    assert kf.tile_config(0, 8192, 8192, torch.float32, "none")["kernel"] == 0
+
+
+def test_argument_validation_returns_before_any_launch(kf):
+    L = kf.lib()
+    P = 0x10000000            # fake, never dereferenced: every case below is rejected on the host
+    ep = kf._Epilogue(None, 0, 1.0, None, 0)
+    rn = kf._RowNorm(1, None, None, 1e-5)
+    call = L.kf_linear_epilogue_rownorm
+    ok_args = dict(X=P, ldx=64, W=P + 0x100000, ldw=64, Y=P + 0x200000, ldy=64, M=32, N=64, K=64, dt=1)
+
+    def run(ep=ep, rn=rn, ws=None, wsb=0, **kw):
+        a = {**ok_args, **kw}
+        return call(a["X"], a["ldx"], a["W"], a["ldw"], a["Y"], a["ldy"], a["M"], a["N"], a["K"], a["dt"],
+                    ctypes.byref(ep), ctypes.byref(rn), ws, wsb, None)
+
+    assert run(M=0) == 0 and run(N=0) == 0                         # empty problem: OK, nothing launched
+    assert run(X=None) == 1 and run(Y=None) == 1 and run(W=None) == 1
+    assert run(M=-1) == 1 and run(dt=7) == 1
+    assert run(ldx=63) == 1 and run(ldy=10) == 1
+    assert run(ep=kf._Epilogue(None, 17, 1.0, None, 0)) == 1
+    assert run(rn=kf._RowNorm(9, None, None, 0.0)) == 1
+    assert run(rn=kf._RowNorm(2, None, None, -1.0)) == 1
+    assert run(ep=kf._Epilogue(None, 0, 1.0, P + 0x300000, 8)) == 1    # residual pitch below N
+    assert run(X=P + 1) == 3                                        # not aligned to the element size
+    assert run(ws=P + 8, wsb=4096, M=4096, N=4096, K=4096, ldx=4096, ldw=4096, ldy=4096) == 3
+    assert run(M=4096, N=4096, K=4096, ldx=4096, ldw=4096, ldy=4096) == 4     # tensor-core path needs ws
+    assert run(M=1 << 31) == 2
+    assert L.kf_row_softmax(None, 8, P, 8, 4, 8, 1, None) == 1
+    assert L.kf_row_layernorm(P, 4, None, None, 1e-5, P, 8, 4, 8, 1, None) == 1
+    assert L.kf_workspace_init(None, 0, None) == 4
+    assert L.kf_check_device_status(None, None, None) == 4
+
+
+def test_host_call_bytes(kf):
+    import torch
+    b = kf.host_call_bytes(256, 512, 128, torch.bfloat16, True, "layernorm")
+    want = 256 * 128 * 2 + 512 * 128 * 2 + 2 * 256 * 512 * 2 + 3 * 1024 + kf.workspace_bytes(256, 512, 128, torch.bfloat16, "layernorm")
+    assert b == want
+
+
+def test_binding_rejects_cpu_tensors(kf):
+    import torch
+    x = torch.zeros(4, 8)
+    with pytest.raises(ValueError):
+        kf.row_softmax(x)
+    with pytest.raises(ValueError):
+        kf.linear_epilogue(x, torch.zeros(3, 8))

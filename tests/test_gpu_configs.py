@@ -1,0 +1,67 @@
+"""GPU parity at the full sizes of the three tensor-core configurations, in the launch configuration
+the bench times: sampled rows against the fp64 oracle (rows are independent, so each sampled row is
+checked over all N columns), plus properties that hold for every row."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2603_12440_b200 import inputs
+from tests.helpers import assert_parity, oracle_of, problem_to_device, to_f64
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def kf():
+    import paper_2603_12440_b200 as m
+    m.binding.lib()
+    return m
+
+
+def _sample_rows(M, n, seed):
+    r = np.random.Generator(np.random.PCG64(seed))
+    return np.unique(np.concatenate([r.choice(M, n, replace=False), [0, 127, 128, M - 1]]))
+
+
+def test_config3_linear_bias_silu_scale_residual(kf):
+    p = inputs.config(3)
+    d = problem_to_device(p)
+    assert kf.tile_config(p.M, p.N, p.K, torch.bfloat16, "none")["kernel"] == 3
+    y = kf.linear_epilogue(d["X"], d["W"], d["bias"], p.act, p.scale, d["residual"])
+    kf.check_device_status()
+    rows = _sample_rows(p.M, 160, 3)
+    r = assert_parity(to_f64(y[torch.from_numpy(rows).cuda()]), oracle_of(inputs.take_rows(p, rows)), "bf16", "C3")
+    assert r["max_ref"] < 8
+
+
+def test_config4_linear_bias_gelu_layernorm(kf):
+    p = inputs.config(4)
+    d = problem_to_device(p)
+    y = kf.linear_epilogue_rownorm(d["X"], d["W"], d["bias"], p.act, p.scale, None, p.norm, d["gamma"], d["beta"], p.eps)
+    kf.check_device_status()
+    rows = _sample_rows(p.M, 160, 4)
+    r = assert_parity(to_f64(y[torch.from_numpy(rows).cuda()]), oracle_of(inputs.take_rows(p, rows)), "bf16", "C4")
+    assert r["max_ref"] < 8
+    # every row: (y - beta) / gamma has mean 0 and variance v / (v + eps) < 1 (v ~ 2e-4 here, eps = 1e-5)
+    z = (y.double() - torch.from_numpy(inputs.to_f64(p.beta)).cuda()) / torch.from_numpy(inputs.to_f64(p.gamma)).cuda()
+    assert float(z.mean(1).abs().max()) < 6e-3
+    var = z.var(1, unbiased=False)
+    assert 0.90 < float(var.min()) and float(var.max()) < 1.0
+
+
+def test_config5_linear_softmax_split_n(kf):
+    p = inputs.config(5)
+    d = problem_to_device(p)
+    y = kf.linear_epilogue_rownorm(d["X"], d["W"], None, "none", 1.0, None, "softmax")
+    kf.check_device_status()
+    rows = _sample_rows(p.M, 96, 5)
+    ref = oracle_of(inputs.take_rows(p, rows))
+    got = to_f64(y[torch.from_numpy(rows).cuda()])
+    assert_parity(got, ref, "bf16", "C5")
+    # outputs are strictly positive with no cancellation: plain element-wise relative error must
+    # also hold wherever the value is representable with full bf16 precision
+    big = ref > 1e-30
+    assert np.max(np.abs(got[big] - ref[big]) / ref[big]) < 1e-2
+    sums = y.double().sum(1)
+    assert float((sums - 1).abs().max()) < 4e-3
+    assert float(y.min()) >= 0

@@ -1,0 +1,225 @@
+"""GPU parity: kf_linear_epilogue and kf_linear_epilogue_rownorm against the fp64 oracle on shapes
+that span several tiles with ragged tails, every activation and row op, both dtypes and all
+kernel families (CUDA-core row-resident, CUDA-core tiled, tcgen05)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import kfo
+from paper_2603_12440_b200 import inputs
+from tests.helpers import assert_parity, oracle_of, problem_to_device, to_device, to_f64
+
+pytestmark = pytest.mark.gpu
+
+ACTS = ["none", "gelu_erf", "gelu_tanh", "silu", "relu", "sigmoid"]
+
+
+@pytest.fixture(scope="module")
+def kf():
+    import paper_2603_12440_b200 as m
+    m.binding.lib()
+    return m
+
+
+def run(kf, p):
+    d = problem_to_device(p)
+    if p.norm == "none":
+        y = kf.linear_epilogue(d["X"], d["W"], d["bias"], p.act, p.scale, d["residual"])
+    else:
+        y = kf.linear_epilogue_rownorm(d["X"], d["W"], d["bias"], p.act, p.scale, d["residual"], p.norm,
+                                       d["gamma"], d["beta"], p.eps)
+    kf.check_device_status()
+    return to_f64(y)
+
+
+def make(dtype, M, N, K, seed, act="none", norm="none", bias=True, res=False, scale=1.0, std=None):
+    std = std if std is not None else 1.0 / np.sqrt(max(K, 1))
+    return inputs.make_problem(f"t{seed}", dtype, M, N, K, seed=seed, std_x=1.0, std_w=std,
+                               bias_std=0.5 if bias else None, residual_std=1.0 if res else None,
+                               gamma_std=0.1 if norm in ("layernorm", "rmsnorm") else None,
+                               beta_std=0.1 if norm == "layernorm" else None, act=act, scale=scale, norm=norm)
+
+
+# ------------------------------------------------------------------------------- fp32 (CUDA cores)
+def test_config1_fp32_full(kf):
+    p = inputs.config(1)
+    assert kf.tile_config(p.M, p.N, p.K, torch.float32, p.norm)["kernel"] == 1
+    r = assert_parity(run(kf, p), oracle_of(p), "f32", "C1")
+    assert r["max_abs"] < 1e-6                      # far inside the 1e-4 gate
+    # the pre-norm values through kf_linear_epilogue (values ~0.06) under the same 1e-4 gate
+    q = inputs.config(1); q.norm = "none"
+    assert_parity(run(kf, q), oracle_of(q), "f32", "C1 pre-norm")
+
+
+@pytest.mark.parametrize("act", ACTS)
+def test_fp32_activations_row_resident(kf, act):
+    p = make("f32", 67, 300, 129, seed=11, act=act, res=True, scale=0.5)
+    assert_parity(run(kf, p), oracle_of(p), "f32", act)
+
+
+@pytest.mark.parametrize("norm", ["softmax", "layernorm", "rmsnorm"])
+@pytest.mark.parametrize("M,N,K", [(1, 1, 1), (5, 7, 3), (33, 256, 64), (300, 257, 100), (17, 1000, 77), (9, 2048, 40),
+                                   (3, 40, 0)])
+def test_fp32_rownorm_row_resident(kf, norm, M, N, K):
+    p = make("f32", M, N, K, seed=12 + N, act="gelu_erf", norm=norm, res=True)
+    assert kf.tile_config(M, N, K, torch.float32, norm)["kernel"] == 1
+    assert_parity(run(kf, p), oracle_of(p), "f32", f"{norm} {M}x{N}x{K}")
+
+
+@pytest.mark.parametrize("norm", ["none", "softmax", "layernorm"])
+def test_fp32_tiled_kernel_and_unfused_rownorm(kf, norm):
+    M, N, K = 130, 2500, 70                         # N > 2048: tiled GEMM, row op as a second in-place kernel
+    p = make("f32", M, N, K, seed=13, act="silu", norm=norm, res=True, scale=0.5)
+    assert kf.tile_config(M, N, K, torch.float32, norm)["kernel"] == 2
+    assert_parity(run(kf, p), oracle_of(p), "f32", f"tiled {norm}")
+    p = make("f32", 1500, 96, 33, seed=14, act="relu")           # tall: tiled kernel without a row op
+    assert kf.tile_config(1500, 96, 33, torch.float32, "none")["kernel"] == 2
+    assert_parity(run(kf, p), oracle_of(p), "f32", "tall")
+
+
+def test_bf16_unaligned_goes_to_cuda_cores(kf):
+    # K not a multiple of 8 rules out TMA; served by the generic kernels in bf16
+    p = make("bf16", 70, 200, 100 + 3, seed=15, act="gelu_erf", norm="softmax", res=True)
+    assert kf.tile_config(p.M, p.N, p.K, torch.bfloat16, "softmax", aligned=False)["kernel"] == 1
+    assert_parity(run(kf, p), oracle_of(p), "bf16", "bf16 simt")
+
+
+# ------------------------------------------------------------------------------- bf16 (tcgen05)
+def test_tc_small_integers_are_bit_exact(kf):
+    """Integer-valued operands make every product and partial sum exact in fp32 and every output
+    exactly representable in bf16: the tensor-core path must reproduce the oracle bit for bit.
+    3 row tiles, 3 column tiles and 4 k-blocks, all with ragged tails."""
+    r = np.random.Generator(np.random.PCG64(21))
+    M, N, K = 300, 520, 200
+    X = inputs.f32_to_bf16_bits(r.integers(-1, 2, (M, K)).astype(np.float32))
+    W = inputs.f32_to_bf16_bits(r.integers(-2, 3, (N, K)).astype(np.float32))
+    assert kf.tile_config(M, N, K, torch.bfloat16, "none")["kernel"] == 3
+    y = kf.linear_epilogue(to_device(X, "bf16"), to_device(W, "bf16"))
+    kf.check_device_status()
+    ref = kfo.linear_epilogue(X, W)
+    assert np.abs(ref).max() <= 256
+    assert np.array_equal(to_f64(y), ref)
+
+
+def test_tc_identity_weight_reproduces_x_bit_exactly(kf):
+    r = np.random.Generator(np.random.PCG64(22))
+    M, K = 1000, 512
+    X = inputs._store(r.standard_normal((M, K)), "bf16")
+    I = inputs._store(np.eye(K), "bf16")
+    assert kf.tile_config(M, K, K, torch.bfloat16, "none")["kernel"] == 3
+    y = kf.linear_epilogue(to_device(X, "bf16"), to_device(I, "bf16"))
+    assert np.array_equal(to_f64(y), inputs.to_f64(X))
+
+
+def test_tc_zero_x_yields_epilogue_of_bias_alone(kf):
+    p = make("bf16", 256, 512, 128, seed=23, act="gelu_erf", norm="softmax", res=False)
+    p.X[:] = 0
+    y = run(kf, p)
+    assert_parity(y, oracle_of(p), "bf16", "zero X")
+    assert np.abs(y - y[0]).max() == 0              # every row is the same function of the bias
+
+
+@pytest.mark.parametrize("act", ACTS)
+def test_tc_activations_with_bias_scale_residual(kf, act):
+    p = make("bf16", 300, 520, 200, seed=24, act=act, res=True, scale=0.5)
+    assert kf.tile_config(p.M, p.N, p.K, torch.bfloat16, "none")["kernel"] == 3
+    assert_parity(run(kf, p), oracle_of(p), "bf16", act)
+
+
+@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (129, 264, 72), (1, 2056, 4104), (700, 8, 8), (257, 1032, 520)])
+def test_tc_shapes(kf, M, N, K):
+    p = make("bf16", M, N, K, seed=25 + M, act="silu", res=True)
+    if kf.tile_config(M, N, K, torch.bfloat16, "none")["kernel"] != 3:
+        pytest.skip("below the tensor-core threshold of the table")
+    assert_parity(run(kf, p), oracle_of(p), "bf16", f"{M}x{N}x{K}")
+
+
+@pytest.mark.parametrize("norm", ["softmax", "layernorm", "rmsnorm"])
+@pytest.mark.parametrize("M,N,K", [(300, 520, 200), (130, 4104, 136), (64, 256, 1024)])
+def test_tc_rownorm_split_n(kf, norm, M, N, K):
+    """Row statistics merged across N-tiles owned by different CTAs (3, 17 and 1 tiles, ragged)."""
+    p = make("bf16", M, N, K, seed=26 + N, act="gelu_erf", norm=norm, res=True)
+    cfg = kf.tile_config(M, N, K, torch.bfloat16, norm)
+    assert cfg["kernel"] == 3 and cfg["row_scheme"] == 2
+    assert_parity(run(kf, p), oracle_of(p), "bf16", f"{norm} {M}x{N}x{K}")
+
+
+def test_tc_layernorm_with_mean_far_from_zero(kf):
+    # sigmoid outputs sit near 0.5 with a small spread: the per-tile shift keeps the deviations exact
+    p = make("bf16", 200, 1536, 256, seed=27, act="sigmoid", norm="layernorm", res=False, std=0.01)
+    assert_parity(run(kf, p), oracle_of(p), "bf16", "ln offset mean")
+
+
+def test_tc_softmax_needs_max_subtraction(kf):
+    """Logits near +90 (constant bias) and logits 8x larger than the benchmark's: exp without the
+    running max would overflow fp32; the oracle stays finite and so must the kernel."""
+    p = make("bf16", 200, 1024, 256, seed=28, norm="softmax", bias=True)
+    p.bias = inputs._store(np.full(p.N, 90.0), "bf16")
+    y = run(kf, p)
+    assert_parity(y, oracle_of(p), "bf16", "bias +90")
+    np.testing.assert_allclose(y.sum(1), 1.0, atol=6e-3)
+    q = inputs.make_problem("big", "bf16", 160, 2048, 1024, seed=29, std_x=2.0, norm="softmax")   # logits ~ N(0, 128^2)
+    assert_parity(run(kf, q), oracle_of(q), "bf16", "huge logits")
+
+
+def test_tc_residual_may_alias_output(kf):
+    p = make("bf16", 300, 520, 200, seed=30, act="silu", res=True)
+    d = problem_to_device(p)
+    out = d["residual"]
+    y = kf.linear_epilogue(d["X"], d["W"], d["bias"], p.act, p.scale, out, out=out)
+    assert y.data_ptr() == out.data_ptr()
+    assert_parity(to_f64(y), oracle_of(p), "bf16", "aliased residual")
+
+
+def test_tc_padded_pitches_and_canaries(kf):
+    """Row pitches larger than the rows; memory between rows and behind the output must stay untouched."""
+    p = make("bf16", 150, 264, 136, seed=31, act="relu", norm="layernorm", res=True)
+    d = problem_to_device(p)
+    def padded(t, extra):
+        big = torch.full((t.shape[0], t.shape[1] + extra), 7.0, dtype=t.dtype, device="cuda")
+        big[:, :t.shape[1]] = t
+        return big, big[:, :t.shape[1]]
+    _, X = padded(d["X"], 8)
+    _, W = padded(d["W"], 16)
+    _, R = padded(d["residual"], 24)
+    ybig, Y = padded(torch.zeros(p.M, p.N, dtype=torch.bfloat16, device="cuda"), 40)
+    kf.linear_epilogue_rownorm(X, W, d["bias"], p.act, p.scale, R, p.norm, d["gamma"], d["beta"], p.eps, out=Y)
+    kf.check_device_status()
+    assert_parity(to_f64(Y), oracle_of(p), "bf16", "padded")
+    assert bool((ybig[:, p.N:] == 7.0).all())
+
+
+def test_tc_deterministic_and_fresh_each_call(kf):
+    p = make("bf16", 300, 2056, 200, seed=32, act="gelu_erf", norm="softmax", res=True)
+    d = problem_to_device(p)
+    args = (d["X"], d["W"], d["bias"], p.act, p.scale, d["residual"], p.norm)
+    y1 = kf.linear_epilogue_rownorm(*args).clone()
+    y2 = kf.linear_epilogue_rownorm(*args)
+    assert torch.equal(y1, y2)
+    d["X"].mul_(-1)                                  # a new input must give a new answer: nothing is cached
+    y3 = kf.linear_epilogue_rownorm(*args)
+    assert not torch.equal(y1, y3)
+
+
+def test_host_buffer_call_matches_device_call(kf):
+    p = make("bf16", 300, 520, 200, seed=33, act="gelu_erf", norm="layernorm", res=True)
+    d = problem_to_device(p)
+    ydev = kf.linear_epilogue_rownorm(d["X"], d["W"], d["bias"], p.act, p.scale, d["residual"], p.norm,
+                                      d["gamma"], d["beta"], p.eps)
+    h = {k: (v.cpu().pin_memory() if v is not None else None) for k, v in d.items()}
+    out = torch.empty(p.M, p.N, dtype=torch.bfloat16).pin_memory()
+    arena = torch.empty(kf.host_call_bytes(p.M, p.N, p.K, torch.bfloat16, True, p.norm), dtype=torch.uint8, device="cuda")
+    kf.linear_epilogue_rownorm_host(h["X"], h["W"], out, arena, h["bias"], p.act, p.scale, h["residual"], p.norm,
+                                    h["gamma"], h["beta"], p.eps)
+    torch.cuda.synchronize()
+    assert torch.equal(out, ydev.cpu())
+
+
+def test_degenerate_sizes(kf):
+    x = torch.zeros(0, 64, dtype=torch.bfloat16, device="cuda")
+    w = torch.zeros(32, 64, dtype=torch.bfloat16, device="cuda")
+    assert kf.linear_epilogue_rownorm(x, w, norm="softmax").shape == (0, 32)
+    one = make("bf16", 40, 1, 16, seed=34, norm="softmax")
+    assert np.all(run(kf, one) == 1.0)
+    ln1 = make("f32", 40, 1, 16, seed=35, norm="layernorm")
+    assert_parity(run(kf, ln1), oracle_of(ln1), "f32", "N=1 layernorm = beta")

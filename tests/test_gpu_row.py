@@ -1,0 +1,100 @@
+"""GPU parity: stand-alone row operators (kf_row_softmax / kf_row_layernorm / kf_row_rmsnorm)
+against the fp64 oracle, element by element, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import kfo
+from paper_2603_12440_b200 import inputs
+from tests.helpers import assert_parity, to_device, to_f64
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def kf():
+    import paper_2603_12440_b200 as m
+    m.binding.lib()
+    return m
+
+
+def _draw(seed, M, N, dtype, std=1.0, shift=0.0):
+    r = np.random.Generator(np.random.PCG64(seed))
+    X = inputs._store(r.standard_normal((M, N)) * std + shift, dtype)
+    g = inputs._store(1 + 0.1 * r.standard_normal(N), dtype)
+    b = inputs._store(0.1 * r.standard_normal(N), dtype)
+    return X, g, b
+
+
+# register-resident shapes (one warp per row up to several warps per row), ragged row counts,
+# and lengths that force the scalar generic kernel (not a multiple of the vector, or too long)
+SHAPES = [(1, 8), (3, 64), (37, 256), (130, 1000), (65, 4096), (19, 4104), (33, 8192), (9, 16384),
+          (5, 32768), (3, 65536), (2, 70000), (7, 1), (11, 13), (6, 1003)]
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("M,N", SHAPES)
+def test_row_ops_match_oracle(kf, dtype, M, N):
+    X, g, b = _draw(100 + N, M, N, dtype, std=2.0, shift=0.5)
+    dX, dg, db = to_device(X, dtype), to_device(g, dtype), to_device(b, dtype)
+    assert_parity(to_f64(kf.row_softmax(dX)), kfo.row_softmax(X), dtype, f"softmax {M}x{N}")
+    assert_parity(to_f64(kf.row_layernorm(dX, dg, db, 1e-5)), kfo.row_layernorm(X, g, b, 1e-5), dtype, f"ln {M}x{N}")
+    assert_parity(to_f64(kf.row_layernorm(dX, None, None, 1e-5)), kfo.row_layernorm(X, None, None, 1e-5), dtype, "ln noaffine")
+    assert_parity(to_f64(kf.row_rmsnorm(dX, dg, 1e-6)), kfo.row_rmsnorm(X, g, 1e-6), dtype, f"rms {M}x{N}")
+    torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_row_ops_in_place_padded_pitch_and_unaligned(kf, dtype):
+    M, N = 50, 2048
+    X, g, b = _draw(7, M, N + 24, dtype)
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    big = to_device(X, dtype)                       # [M, N+24]
+    view = big[:, :N]                               # pitch N+24: still 16-byte friendly
+    ref = kfo.row_layernorm(np.ascontiguousarray(X[:, :N]), np.ascontiguousarray(g[:N]), np.ascontiguousarray(b[:N]), 1e-5)
+    dg, db = to_device(np.ascontiguousarray(g[:N]), dtype), to_device(np.ascontiguousarray(b[:N]), dtype)
+    canary = big[:, N:].clone()
+    out = kf.row_layernorm(view, dg, db, 1e-5, out=view)          # in place
+    assert out.data_ptr() == view.data_ptr()
+    assert_parity(to_f64(view), ref, dtype, "in-place ln")
+    assert torch.equal(big[:, N:], canary), "wrote outside the row"
+    # unaligned base pointer (offset by one element) -> generic kernel
+    flat = torch.zeros(M * N + 1, dtype=tdt, device="cuda")
+    flat[1:] = to_device(np.ascontiguousarray(X[:, :N]), dtype).reshape(-1)
+    xu = flat[1:].view(M, N)
+    assert xu.data_ptr() % 16 != 0
+    ref_sm = kfo.row_softmax(np.ascontiguousarray(X[:, :N]))
+    assert_parity(to_f64(kf.row_softmax(xu)), ref_sm, dtype, "unaligned softmax")
+
+
+def test_softmax_large_magnitude_and_invariants(kf):
+    r = np.random.Generator(np.random.PCG64(3))
+    a = (r.standard_normal((64, 4096)) * 30 + 500).astype(np.float32)      # exp(a) overflows fp32
+    y = to_f64(kf.row_softmax(to_device(a, "f32")))
+    assert_parity(y, kfo.row_softmax(a), "f32", "large logits")
+    np.testing.assert_allclose(y.sum(1), 1.0, atol=1e-5)
+    ab = inputs._store(r.standard_normal((64, 4096)) * 3, "bf16")
+    yb = to_f64(kf.row_softmax(to_device(ab, "bf16")))
+    np.testing.assert_allclose(yb.sum(1), 1.0, atol=4e-3)                  # bf16 output rounding only
+    eq = to_f64(kf.row_softmax(torch.full((5, 512), 2.5, device="cuda")))
+    assert np.all(eq == 1.0 / 512)
+
+
+def test_config2_full_size_properties_and_sampled_rows(kf):
+    """bf16 row LayerNorm [16384, 4096] in the launch configuration the bench times: sampled rows
+    against the oracle, every row against the invariants that hold at any size."""
+    p = inputs.config(2)
+    dX, dg, db = to_device(p.X, "bf16"), to_device(p.gamma, "bf16"), to_device(p.beta, "bf16")
+    y = kf.row_layernorm(dX, dg, db, p.eps)
+    torch.cuda.synchronize()
+    rows = np.random.Generator(np.random.PCG64(5)).choice(p.M, 512, replace=False)
+    rows = np.concatenate([rows, [0, p.M - 1]])
+    ref = kfo.row_layernorm(np.ascontiguousarray(p.X[rows]), p.gamma, p.beta, p.eps)
+    assert_parity(to_f64(y[torch.from_numpy(rows).cuda()]), ref, "bf16", "C2 sampled rows")
+    # whole tensor: (y - beta) / gamma has row mean ~ 0 and row variance ~ v / (v + eps) ~ 1
+    g64 = torch.from_numpy(inputs.to_f64(p.gamma)).cuda()
+    b64 = torch.from_numpy(inputs.to_f64(p.beta)).cuda()
+    z = (y.double() - b64) / g64
+    assert float(z.mean(1).abs().max()) < 5e-3
+    assert float((z.var(1, unbiased=False) - 1).abs().max()) < 2e-2
+    assert y.is_contiguous() and y.shape == (p.M, p.N)
