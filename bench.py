@@ -1,0 +1,349 @@
+#!/usr/bin/env python
+"""Benchmark of the fused linear + epilogue + row-norm path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl kf|reference] [--no-configs]
+
+A step is one call of ``kf_linear_epilogue_rownorm`` on the headline workload C4 (bf16
+X[4096,2048] . W[8192,2048]^T + bias -> GELU(erf) -> row LayerNorm over all 8192 outputs): operand
+fetch, tcgen05 main loop, element-wise epilogue, split-N row statistics, normalise + store.  Inputs
+are resident in HBM; L2 is flushed between steps (outside the timed events).  ``value`` is the
+whole-job TFLOP/s (2*M*N*K per step and rank, max step time over ranks).  With N > 1 every rank runs
+an independent replica of the same workload (the path has no exchange step).  The other four
+configurations are timed the same way and reported under ``per_config``.
+
+``--impl reference`` times the fp64 CPU oracle on a bounded row sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+METRIC = "fused linear+epilogue+row-norm TFLOP/s (bf16, fp32 accumulate), 1 GPU"
+WORKLOAD = "C4: bf16 X[4096,2048] W[8192,2048] bias+GELU(erf)+row LayerNorm(N=8192), seed 3"
+NOMINAL_TFLOPS, NOMINAL_GBS = 2250.0, 8000.0
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    f = ROOT / "MEASURED_PEAKS.json"
+    if f.exists():
+        try:
+            d = json.loads(f.read_text())
+            return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+        except Exception:
+            pass
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ------------------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period: float = 0.05):
+        self.index, self.period = index, period
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._nv = None
+
+    def _loop(self):
+        nv = self._nv
+        names = {nv.nvmlClocksThrottleReasonHwSlowdown: "hw_slowdown",
+                 nv.nvmlClocksThrottleReasonHwThermalSlowdown: "hw_thermal_slowdown",
+                 nv.nvmlClocksThrottleReasonSwThermalSlowdown: "sw_thermal_slowdown",
+                 nv.nvmlClocksThrottleReasonSwPowerCap: "sw_power_cap"}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def __enter__(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        s = sorted(self.samples)
+        med = s[len(s) // 2] if s else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(s)}
+
+
+# ------------------------------------------------------------------------------------------ kf arm
+def device_problem(p):
+    from paper_2603_12440_b200 import inputs
+    return inputs.problem_to_torch(p, "cuda")
+
+
+def make_call(kf, p, d):
+    """A zero-argument callable that issues the C-ABI call of problem p on device tensors d."""
+    import torch
+    tdt = torch.bfloat16 if p.dtype == "bf16" else torch.float32
+    out = torch.empty((p.M, p.N), dtype=tdt, device="cuda")
+    if p.call == "row_layernorm":
+        return (lambda: kf.row_layernorm(d["X"], d["gamma"], d["beta"], p.eps, out=out)), out
+    if p.call == "linear_epilogue":
+        return (lambda: kf.linear_epilogue(d["X"], d["W"], d["bias"], p.act, p.scale, d["residual"], out=out)), out
+    return (lambda: kf.linear_epilogue_rownorm(d["X"], d["W"], d["bias"], p.act, p.scale, d["residual"], p.norm,
+                                               d["gamma"], d["beta"], p.eps, out=out)), out
+
+
+def time_steps(call, steps, warmup, flush, split=None):
+    """Per-step CUDA-event timing on the current stream with an L2 flush before every step.
+    Returns (list of ms, list of ms up to the split event or None)."""
+    import torch
+    for _ in range(warmup):
+        flush()
+        call()
+    torch.cuda.synchronize()
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    mids = [torch.cuda.Event(enable_timing=True) for _ in range(steps)] if split else None
+    for i in range(steps):
+        flush()
+        if split:
+            mids[i].record()                   # materialise the handle before handing it to the library
+            split(mids[i])
+        starts[i].record()
+        call()
+        ends[i].record()
+    if split:
+        split(None)
+    torch.cuda.synchronize()
+    total = [s.elapsed_time(e) for s, e in zip(starts, ends)]
+    main = [s.elapsed_time(m) for s, m in zip(starts, mids)] if split else None
+    return total, main
+
+
+def median(v):
+    s = sorted(v)
+    return s[len(s) // 2]
+
+
+def run_kf(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2603_12440_b200 as kf
+    from paper_2603_12440_b200 import inputs
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the kf path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    kf.binding.lib()                                        # fail loudly if the CUDA library is missing
+    peaks, peak_src = load_peaks()
+
+    flush_buf = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")     # 4x the 126 MB L2
+
+    def flush():
+        flush_buf.fill_(1)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---------------------------------------------------------------- headline workload
+    p = inputs.config(4)
+    d = device_problem(p)
+    call, out = make_call(kf, p, d)
+    cfg = kf.tile_config(p.M, p.N, p.K, torch.bfloat16, p.norm)
+    barrier()
+    with ClockSampler(local) as clk:
+        barrier()
+        total_ms, main_ms = time_steps(call, args.steps, args.warmup, flush, kf.profile_set_split_event)
+        barrier()
+    kf.check_device_status()
+    ms = sum(total_ms) / len(total_ms)
+    t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_max = float(t.item())
+    tflops = world * p.flops / (ms_max * 1e-3) / 1e12
+
+    main_avg = sum(main_ms) / len(main_ms)
+    achieved = p.flops / (main_avg * 1e-3) / 1e12
+    roofline = {"bound": "tensor", "kernel": "tc_linear_kernel (tcgen05 GEMM + fused epilogue + row partials)",
+                "achieved": round(achieved, 2), "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": round(achieved / peaks["bf16_tflops"], 4), "peak_source": f"{peak_src} burst cuBLAS bf16",
+                "frac_of_sustained": round(achieved / peaks["bf16_tflops_sustained"], 4),
+                "frac_of_nominal_2250": round(achieved / NOMINAL_TFLOPS, 4),
+                "kernel_ms": round(main_avg, 5), "finish_kernel_ms": round(ms - main_avg, 5),
+                "traffic": TRAFFIC.get("c4_main")}
+
+    # ---------------------------------------------------------------- end to end from host buffers
+    e2e = None
+    if rank == 0 or world > 1:
+        h = {k: (v.cpu().pin_memory() if v is not None else None) for k, v in d.items()}
+        hout = torch.empty((p.M, p.N), dtype=torch.bfloat16).pin_memory()
+        arena = torch.empty(kf.host_call_bytes(p.M, p.N, p.K, torch.bfloat16, False, p.norm), dtype=torch.uint8,
+                            device="cuda")
+
+        def host_call():
+            kf.linear_epilogue_rownorm_host(h["X"], h["W"], hout, arena, h["bias"], p.act, p.scale, None, p.norm,
+                                            h["gamma"], h["beta"], p.eps)
+        e_steps = max(3, min(args.steps, 10))
+        barrier()
+        e_ms, _ = time_steps(host_call, e_steps, 3, flush)
+        barrier()
+        te = torch.tensor([sum(e_ms) / len(e_ms)], dtype=torch.float64, device="cuda")
+        if world > 1:
+            dist.all_reduce(te, op=dist.ReduceOp.MAX)
+        h2d = sum(v.numel() * v.element_size() for v in (h["X"], h["W"], h["bias"], h["gamma"], h["beta"]))
+        e2e = {"value": round(world * p.flops / (float(te.item()) * 1e-3) / 1e12, 3), "unit": "TFLOP/s",
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(hout.numel() * 2),
+               "ms_per_step": round(float(te.item()), 4), "steps": e_steps,
+               "api": "kf_linear_epilogue_rownorm_host (pinned host buffers in, pinned host Y out)"}
+        del arena, h, hout
+
+    # ---------------------------------------------------------------- the other configurations
+    per_config = {}
+    launches = args.steps * 2
+    if rank == 0 and not args.no_configs:
+        for idx in (1, 2, 3, 4, 5):
+            q = p if idx == 4 else inputs.config(idx)
+            dq = d if idx == 4 else device_problem(q)
+            cq, _ = make_call(kf, q, dq)
+            steps = max(5, min(args.steps, 20))
+            tms, _ = time_steps(cq, steps, 3, flush)
+            m = median(tms)
+            ent = {"call": q.call, "dtype": q.dtype, "M": q.M, "N": q.N, "K": q.K, "ms_median": round(m, 5),
+                   "ms_min": round(min(tms), 5), "GB/s": round(q.algorithmic_bytes / (m * 1e-3) / 1e9, 1),
+                   "frac_hbm_measured": round(q.algorithmic_bytes / (m * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
+                   "frac_hbm_nominal_8000": round(q.algorithmic_bytes / (m * 1e-3) / 1e9 / NOMINAL_GBS, 4)}
+            if q.K:
+                tf = q.flops / (m * 1e-3) / 1e12
+                ent.update({"TFLOP/s": round(tf, 2), "frac_tensor_measured_burst": round(tf / peaks["bf16_tflops"], 4),
+                            "frac_tensor_nominal_2250": round(tf / NOMINAL_TFLOPS, 4)})
+                tc = kf.tile_config(q.M, q.N, q.K, torch.bfloat16 if q.dtype == "bf16" else torch.float32, q.norm)
+                ent["tile"] = {k: tc[k] for k in ("kernel", "bm", "bn", "bk", "stages", "cta_group", "row_scheme", "grid")}
+            per_config[q.name] = ent
+            if idx != 4:
+                del dq, cq
+                torch.cuda.empty_cache()
+        kf.check_device_status()
+
+    # ---------------------------------------------------------------- CPU baseline (oracle, rank 0, N == 1)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        cpu = cpu_baseline_sample(p)
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": round(tflops, 2), "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": round(ms_max, 5), "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": WORKLOAD, "M": p.M, "N": p.N, "K": p.K, "epilogue": "bias+gelu_erf",
+                           "rownorm": "layernorm", "parallelism": "replicas only" if world > 1 else "1 gpu",
+                           "l2": "flushed between steps (512 MiB write, outside the timed events)",
+                           "tile": {k: cfg[k] for k in ("kernel", "bm", "bn", "bk", "stages", "cta_group",
+                                                        "epilogue_warps", "row_scheme", "grid")}},
+                "clocks": clk.summary(), "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
+                "cpu_baseline": cpu, "per_config": per_config,
+                "frac_of_measured_burst": round(tflops / world / peaks["bf16_tflops"], 4),
+                "frac_of_nominal_2250": round(tflops / world / NOMINAL_TFLOPS, 4)}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# DRAM bytes per launch from ncu captures (dram__bytes_read.sum + dram__bytes_write.sum); see profiles/
+TRAFFIC = {"c4_main": None}
+
+
+# ------------------------------------------------------------------------------------------ CPU arms
+def cpu_baseline_sample(p, rows: int = 768):
+    """The oracle as it stands on a bounded sample (the first `rows` rows) of the workload."""
+    from oracle import kfo
+    from paper_2603_12440_b200 import inputs
+    q = inputs.take_rows(p, list(range(rows)))
+    t0 = time.perf_counter()
+    kfo.linear_epilogue_rownorm(q.X, q.W, q.bias, q.act, q.scale, q.residual, q.norm, q.gamma, q.beta, q.eps)
+    dt = time.perf_counter() - t0
+    return {"value": round(q.flops / dt / 1e12, 6), "unit": "TFLOP/s", "cores": kfo.threads(), "kind": "oracle",
+            "sample": f"first {rows} of {p.M} rows of C4, all {p.N} columns, fp64, {dt:.2f} s wall",
+            "host_cpus": os.cpu_count()}
+
+
+def run_reference(args):
+    """The reference arm of this tier is the fp64 CPU oracle, timed on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import kfo
+    from paper_2603_12440_b200 import inputs
+    p = inputs.config(4)
+    rows = 128
+    q = inputs.take_rows(p, list(range(rows)))
+
+    def step():
+        kfo.linear_epilogue_rownorm(q.X, q.W, q.bias, q.act, q.scale, q.residual, q.norm, q.gamma, q.beta, q.eps)
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / args.steps
+    val = round(q.flops / dt / 1e12, 6)
+    sample = f"each step = first {rows} of {p.M} rows of C4, all {p.N} columns, fp64"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s",
+        "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": round(dt * 1e3, 3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "M": p.M, "N": p.N, "K": p.K, "sample": sample},
+        "cpu_baseline": {"value": val, "unit": "TFLOP/s", "kind": "oracle", "cores": kfo.threads(), "sample": sample},
+        "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="kf", choices=["kf", "reference"])
+    ap.add_argument("--no-configs", action="store_true", help="skip the per-configuration table")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "kf" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_kf(args)
+
+
+if __name__ == "__main__":
+    main()

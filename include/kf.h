@@ -166,6 +166,13 @@ kf_status kf_check_device_status(void *ws, void *stream, uint32_t *detail);
 kf_status kf_tile_config_query(int64_t M, int64_t N, int64_t K, kf_dtype dt, kf_norm norm,
                                int aligned, kf_tile_config *out);
 
+/* Profiling aid (the paper feeds per-kernel profiler figures back into its search, Appendix B.3):
+ * while `event` (a cudaEvent_t, or NULL to switch off) is set, every tensor-core linear call
+ * records it on the call's stream right after its main GEMM kernel, before any finishing pass, so
+ * a caller that brackets the call with its own events can time the two kernels separately.
+ * Process-wide, not thread-safe; leave it off outside benchmarks. */
+kf_status kf_profile_set_split_event(void *event);
+
 const char *kf_status_string(kf_status s);
 
 /* Library version as major * 10000 + minor * 100 + patch. */

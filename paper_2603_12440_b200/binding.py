@@ -76,6 +76,8 @@ def lib() -> ctypes.CDLL:
     L.kf_workspace_init.argtypes = [vp, sz, vp]
     L.kf_check_device_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
     L.kf_tile_config_query.argtypes = [i64, i64, i64, ci, ci, ci, ctypes.POINTER(TileConfig)]
+    L.kf_profile_set_split_event.argtypes = [vp]
+    L.kf_profile_set_split_event.restype = ci
     L.kf_status_string.argtypes = [ci]
     L.kf_status_string.restype = ctypes.c_char_p
     L.kf_version.argtypes = []
@@ -148,6 +150,13 @@ def check_device_status(ws: Optional[torch.Tensor] = None, stream=None):
     st = lib().kf_check_device_status(ws.data_ptr(), _stream(stream), ctypes.byref(detail))
     if st != KF_OK:
         raise KfError(st, f"device status (detail 0x{detail.value:x})")
+
+
+def profile_set_split_event(event: Optional[torch.cuda.Event]):
+    """Record ``event`` between the GEMM kernel and the finishing pass of later tensor-core calls
+    (``None`` switches it off).  The event must have been created with ``enable_timing=True`` and
+    recorded once before, so that its CUDA handle exists."""
+    _check(lib().kf_profile_set_split_event(None if event is None else event.cuda_event), "kf_profile_set_split_event")
 
 
 def tile_config(M: int, N: int, K: int, dtype, norm: str = "none", aligned: bool = True) -> dict:

@@ -37,8 +37,7 @@ kf_status resolve(long long M, long long N, long long K, int dt, int norm, bool 
     if (M == 0 || N == 0) return KF_OK;
     const Override& ov = env_override();
     const bool tc_ok = dt == KF_BF16 && aligned && K > 0 && K % 8 == 0 && N % 8 == 0;
-    const double flops = 2.0 * (double)M * (double)N * (double)K;
-    bool use_tc = tc_ok && (flops >= 16.0e6 || (norm != KF_NORM_NONE && !simt_row_resident_ok(N)));
+    bool use_tc = tc_ok;
     if (ov.kernel == 3 && tc_ok) use_tc = true;
     if ((ov.kernel == 1 || ov.kernel == 2) &&
         (norm == KF_NORM_NONE || dt == KF_F32 || simt_row_resident_ok(N)))
@@ -276,6 +275,11 @@ const char* kf_status_string(kf_status s) {
     case KF_ERR_TIMEOUT: return "KF_ERR_TIMEOUT";
     default: return "KF_ERR_UNKNOWN";
     }
+}
+
+kf_status kf_profile_set_split_event(void* event) {
+    tc_set_split_event(static_cast<cudaEvent_t>(event));
+    return KF_OK;
 }
 
 int kf_version(void) { return 100; }

@@ -646,6 +646,9 @@ int sm_count() {
 
 }  // namespace
 
+static cudaEvent_t g_split_event = nullptr;
+void tc_set_split_event(cudaEvent_t ev) { g_split_event = ev; }
+
 void tc_tile_shape(int* bm, int* bn, int* bk, int* stages, int* epi_warps) {
     *bm = BM; *bn = BN; *bk = BK; *stages = kStages; *epi_warps = kEpiWarps;
 }
@@ -702,6 +705,7 @@ kf_status launch_tc_linear(const void* X, long long ldx, const void* W, long lon
     if (grid_out) *grid_out = grid;
     tc_linear_kernel<<<grid, kThreads, kSmemAlloc, st>>>(tmX, tmW, tmY, p);
     if (cudaGetLastError() != cudaSuccess) return KF_ERR_CUDA;
+    if (g_split_event && cudaEventRecord(g_split_event, st) != cudaSuccess) return KF_ERR_CUDA;
 
     if (rn.norm != KF_NORM_NONE) {
         const size_t sm = (size_t)p.tiles_n * 2 * sizeof(float);

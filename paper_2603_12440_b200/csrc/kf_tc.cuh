@@ -15,4 +15,7 @@ kf_status launch_tc_linear(const void* X, long long ldx, const void* W, long lon
                            long long M, long long N, long long K, const EpilogueParams& ep, const RowNormParams& rn,
                            void* ws, int grid_override, cudaStream_t st, int* grid_out);
 
+// profiling aid: event recorded between the GEMM kernel and the finishing kernel (nullptr = off)
+void tc_set_split_event(cudaEvent_t ev);
+
 }  // namespace kf

@@ -151,3 +151,18 @@ def take_rows(p: Problem, rows) -> Problem:
     if p.residual is not None:
         q.residual = np.ascontiguousarray(p.residual[rows])
     return q
+
+
+def to_torch(a, dtype: str, device="cuda"):
+    """numpy float32 array, or uint16 bf16 bit patterns, -> torch tensor of that dtype on `device`."""
+    import torch
+    if a is None:
+        return None
+    if dtype == "bf16":
+        return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).view(torch.bfloat16).to(device)
+    return torch.from_numpy(np.ascontiguousarray(a)).to(device)
+
+
+def problem_to_torch(p: Problem, device="cuda") -> dict:
+    """The tensors of a problem on `device`, keyed X, W, bias, residual, gamma, beta (absent ones None)."""
+    return {k: to_torch(getattr(p, k), p.dtype, device) for k in ("X", "W", "bias", "residual", "gamma", "beta")}

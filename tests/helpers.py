@@ -13,13 +13,7 @@ import torch
 from paper_2603_12440_b200 import inputs
 
 
-def to_device(a, dtype: str, device="cuda"):
-    """numpy float32 array, or uint16 bf16 bit patterns, -> CUDA tensor of that dtype."""
-    if a is None:
-        return None
-    if dtype == "bf16":
-        return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).view(torch.bfloat16).to(device)
-    return torch.from_numpy(np.ascontiguousarray(a)).to(device)
+to_device = inputs.to_torch
 
 
 def to_f64(t: torch.Tensor) -> np.ndarray:
@@ -55,13 +49,11 @@ def assert_parity(got: np.ndarray, ref: np.ndarray, dtype: str, what: str = ""):
     return r
 
 
-def problem_to_device(p):
-    d = p.dtype
-    return {k: to_device(getattr(p, k), d) for k in ("X", "W", "bias", "residual", "gamma", "beta")}
+problem_to_device = inputs.problem_to_torch
 
 
 def oracle_of(p):
     from oracle import kfo
-    if p.K == 0:
+    if p.W is None:
         return kfo.row_norm(p.X, p.norm, p.gamma, p.beta, p.eps)
     return kfo.linear_epilogue_rownorm(p.X, p.W, p.bias, p.act, p.scale, p.residual, p.norm, p.gamma, p.beta, p.eps)
