@@ -48,7 +48,7 @@ def load_peaks():
 class ClockSampler:
     """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
 
-    def __init__(self, index: int, period: float = 0.05):
+    def __init__(self, index: int, period: float = 0.005):
         self.index, self.period = index, period
         self.samples, self.reasons = [], set()
         self.max_mhz = None
@@ -175,6 +175,18 @@ def run_kf(args):
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
+
+    if args.only:
+        # one configuration alone, for profiler captures: few launches, nothing else on the device
+        idx = int(args.only.lower().lstrip("c"))
+        q = inputs.config(idx)
+        dq = device_problem(q)
+        cq, _ = make_call(kf, q, dq)
+        tms, _ = time_steps(cq, args.steps, args.warmup, flush)
+        kf.check_device_status()
+        print(json.dumps({"only": q.name, "steps": args.steps, "ms_median": round(median(tms), 5),
+                          "ms_min": round(min(tms), 5)}))
+        return
 
     # ---------------------------------------------------------------- headline workload
     p = inputs.config(4)
@@ -332,13 +344,15 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="kf", choices=["kf", "reference"])
     ap.add_argument("--no-configs", action="store_true", help="skip the per-configuration table")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
+    ap.add_argument("--only", default=None, help="time one configuration alone (c1..c5), e.g. under a profiler")
     args = ap.parse_args()
-    args.warmup = max(args.warmup, 3) if args.impl == "kf" else args.warmup
+    if args.impl == "kf" and not args.only:
+        args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
         run_reference(args)
     else:
