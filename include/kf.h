@@ -50,7 +50,8 @@ typedef enum {
     KF_ERR_ALIGNMENT = 3,     /* pointer not aligned to its element size / workspace not 256-byte aligned */
     KF_ERR_WORKSPACE = 4,     /* ws is NULL or smaller than kf_workspace_bytes */
     KF_ERR_CUDA = 5,          /* a CUDA runtime / driver call failed (launch, tensor-map encode) */
-    KF_ERR_TIMEOUT = 6        /* device status word: a bounded wait inside a kernel gave up */
+    KF_ERR_TIMEOUT = 6,       /* device status word: a bounded wait inside a kernel gave up */
+    KF_ERR_SCRATCH_LIMIT = 7  /* kf_linear_epilogue_rownorm_noalloc: problem needs more than the built-in scratch */
 } kf_status;
 
 typedef enum { KF_F32 = 0, KF_BF16 = 1 } kf_dtype;
@@ -148,6 +149,42 @@ kf_status kf_linear_epilogue_rownorm_host(const void *X, const void *W, void *Y,
                                           size_t dev_bytes, void *stream);
 size_t kf_host_call_bytes(int64_t M, int64_t N, int64_t K, kf_dtype dt, int has_residual,
                           kf_norm norm);
+
+/*
+ * Allocation-free form of kf_linear_epilogue_rownorm.  (The paper has no counterpart: this exists
+ * for the callers described next.)
+ *
+ * Who needs it: code that is handed its input and output buffers but has no way to obtain device
+ * scratch of its own -- a plug-in running inside a host application whose memory pool it may not
+ * touch, a real-time or safety-reviewed service where every cudaMalloc / cudaFree after start-up is
+ * forbidden because it synchronises the device and can fail or fragment, or a client that only
+ * holds externally shared buffers.  Such a caller cannot provide the `ws` argument of the normal
+ * form.  This form takes none: the status block and the per-row partial statistics live in an
+ * array compiled into the library's device image.
+ *
+ * Same arguments, results and kernels as kf_linear_epilogue_rownorm, minus ws / ws_bytes.
+ *   - Limit: kf_workspace_bytes(M,N,K,dt,norm) must not exceed 4 MiB + 256 bytes, i.e. a bf16
+ *     row-norm may span at most 2048 output tiles of 128 x 256 (ceil(M/128) * ceil(N/256)).  Larger
+ *     problems return KF_ERR_SCRATCH_LIMIT and launch nothing.  Calls without a row-norm and fp32
+ *     calls need only the status block and are never rejected for size.
+ *   - Every device that loads the library holds the 4 MiB array until the process exits.
+ *   - The call performs no cudaMalloc / cudaFree and calls no allocating routine.  The first call
+ *     on each device looks the array's device address up (cudaGetSymbolAddress, with that device
+ *     current, which may load the module); make that first call before starting any stream capture.
+ *   - The array is shared by all calls on a device and keeps the previous call's contents; each call
+ *     clears the status block on `stream` and overwrites every partial it later reads.  Two calls of
+ *     this form that overlap on the GPU (different streams, or concurrent host threads) race on the
+ *     array: serialise them on one stream.
+ *   - device_status: NULL, or a HOST pointer to two uint32.  When given, the call waits for `stream`
+ *     after launching, copies the status block's {status, detail} words there and returns
+ *     KF_ERR_TIMEOUT if a bounded on-device wait gave up.  With NULL the call stays asynchronous
+ *     and a device-side time-out goes unreported.
+ */
+kf_status kf_linear_epilogue_rownorm_noalloc(const void *X, int64_t ldx, const void *W, int64_t ldw,
+                                             void *Y, int64_t ldy, int64_t M, int64_t N, int64_t K,
+                                             kf_dtype dt, const kf_epilogue *ep,
+                                             const kf_rownorm *rn, void *stream,
+                                             uint32_t *device_status);
 
 /* Bytes of `ws` the two linear calls need for this shape (always >= 256). */
 size_t kf_workspace_bytes(int64_t M, int64_t N, int64_t K, kf_dtype dt, kf_norm norm);

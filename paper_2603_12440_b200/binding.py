@@ -69,6 +69,9 @@ def lib() -> ctypes.CDLL:
     L.kf_row_layernorm.argtypes = [vp, i64, vp, vp, cf, vp, i64, i64, i64, ci, vp]
     L.kf_row_rmsnorm.argtypes = [vp, i64, vp, cf, vp, i64, i64, i64, ci, vp]
     L.kf_linear_epilogue_rownorm_host.argtypes = [vp, vp, vp, i64, i64, i64, ci, ep, rn, vp, sz, vp]
+    L.kf_linear_epilogue_rownorm_noalloc.argtypes = [vp, i64, vp, i64, vp, i64, i64, i64, i64, ci, ep, rn, vp,
+                                                     ctypes.POINTER(ctypes.c_uint32)]
+    L.kf_linear_epilogue_rownorm_noalloc.restype = ci
     L.kf_host_call_bytes.argtypes = [i64, i64, i64, ci, ci, ci]
     L.kf_host_call_bytes.restype = sz
     L.kf_workspace_bytes.argtypes = [i64, i64, i64, ci, ci]
@@ -196,6 +199,41 @@ def linear_epilogue_rownorm(X, W, bias=None, act="none", scale=1.0, residual=Non
     st = L.kf_linear_epilogue_rownorm(px, ldx, pw, ldw, py, ldy, M, N, K, DTYPE[X.dtype], ctypes.byref(ep),
                                       ctypes.byref(rn), ws.data_ptr(), ws.numel(), _stream(stream))
     _check(st, "kf_linear_epilogue_rownorm")
+    return out
+
+
+def linear_epilogue_rownorm_noalloc(X, W, out, bias=None, act="none", scale=1.0, residual=None, norm="none",
+                                    gamma=None, beta=None, eps=1e-5, stream=None, wait=False) -> torch.Tensor:
+    """``kf_linear_epilogue_rownorm_noalloc``: the fused call for callers that cannot provide scratch.
+
+    Nothing is allocated here either: ``out`` must be given, and the library uses the scratch array
+    built into its device image (row-norm problems of at most 2048 output tiles; larger ones raise
+    ``KfError`` with status 7).  Calls that overlap on the GPU race on that array, so keep them on one
+    stream.  ``wait=True`` blocks until the stream has finished and raises if a kernel reported a
+    time-out; otherwise the call is asynchronous like the others."""
+    L = lib()
+    if X.dtype not in DTYPE or W.dtype != X.dtype:
+        raise ValueError("X and W must both be float32 or both bfloat16")
+    M, K = X.shape
+    N, K2 = W.shape
+    if K2 != K:
+        raise ValueError("X is [M,K] and W is [N,K]")
+    if out is None or out.dtype != X.dtype or tuple(out.shape) != (M, N):
+        raise ValueError("out must be a preallocated [M,N] tensor of the dtype of X")
+    px, ldx = _mat(X, "X")
+    pw, ldw = _mat(W, "W")
+    py, ldy = _mat(out, "out")
+    ep = _Epilogue(_vec(bias, N, X.dtype, "bias"), ACT[act], float(scale), None, 0)
+    if residual is not None:
+        if residual.dtype != X.dtype or tuple(residual.shape) != (M, N):
+            raise ValueError("residual must be [M,N] of the dtype of X")
+        pr, ldr = _mat(residual, "residual")
+        ep.residual, ep.ldr = pr, ldr
+    rn = _RowNorm(NORM[norm], _vec(gamma, N, X.dtype, "gamma"), _vec(beta, N, X.dtype, "beta"), float(eps))
+    status = (ctypes.c_uint32 * 2)(0, 0)
+    st = L.kf_linear_epilogue_rownorm_noalloc(px, ldx, pw, ldw, py, ldy, M, N, K, DTYPE[X.dtype], ctypes.byref(ep),
+                                              ctypes.byref(rn), _stream(stream), status if wait else None)
+    _check(st, "kf_linear_epilogue_rownorm_noalloc")
     return out
 
 

@@ -255,6 +255,32 @@ kf_status kf_linear_epilogue_rownorm_host(const void* X, const void* W, void* Y,
     return KF_OK;
 }
 
+kf_status kf_linear_epilogue_rownorm_noalloc(const void* X, int64_t ldx, const void* W, int64_t ldw, void* Y,
+                                             int64_t ldy, int64_t M, int64_t N, int64_t K, kf_dtype dt,
+                                             const kf_epilogue* ep, const kf_rownorm* rn, void* stream,
+                                             uint32_t* device_status) {
+    if (device_status) device_status[0] = device_status[1] = 0;
+    if (M > 0 && N > 0 && M < (1ll << 31) && N < (1ll << 31) &&
+        kf_workspace_bytes(M, N, K, dt, rn ? (kf_norm)rn->norm : KF_NORM_NONE) > tc_static_scratch_bytes())
+        return KF_ERR_SCRATCH_LIMIT;                       // host-side check, nothing launched
+    if (M <= 0 || N <= 0)                                  // empty or invalid: same answers as the ws form
+        return kf_linear_epilogue_rownorm(X, ldx, W, ldw, Y, ldy, M, N, K, dt, ep, rn, nullptr, 0, stream);
+    void* scratch = nullptr;
+    kf_status s = tc_static_scratch(&scratch);
+    if (s != KF_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // the array keeps whatever the previous call left: only the status block has to start at zero
+    if (cudaMemsetAsync(scratch, 0, kStatusBytes, st) != cudaSuccess) return KF_ERR_CUDA;
+    s = kf_linear_epilogue_rownorm(X, ldx, W, ldw, Y, ldy, M, N, K, dt, ep, rn, scratch, tc_static_scratch_bytes(),
+                                   stream);
+    if (s != KF_OK || !device_status) return s;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return KF_ERR_CUDA;
+    if (cudaMemcpy(device_status, scratch, 2 * sizeof(uint32_t), cudaMemcpyDeviceToHost) != cudaSuccess)
+        return KF_ERR_CUDA;
+    return device_status[0] == 0 ? KF_OK : (device_status[0] <= (uint32_t)KF_ERR_TIMEOUT ? (kf_status)device_status[0]
+                                                                                          : KF_ERR_CUDA);
+}
+
 kf_status kf_tile_config_query(int64_t M, int64_t N, int64_t K, kf_dtype dt, kf_norm norm, int aligned,
                                kf_tile_config* out) {
     if (!out) return KF_ERR_INVALID_ARG;
@@ -273,6 +299,7 @@ const char* kf_status_string(kf_status s) {
     case KF_ERR_WORKSPACE: return "KF_ERR_WORKSPACE";
     case KF_ERR_CUDA: return "KF_ERR_CUDA";
     case KF_ERR_TIMEOUT: return "KF_ERR_TIMEOUT";
+    case KF_ERR_SCRATCH_LIMIT: return "KF_ERR_SCRATCH_LIMIT";
     default: return "KF_ERR_UNKNOWN";
     }
 }

@@ -646,6 +646,31 @@ int sm_count() {
 
 }  // namespace
 
+// ---- built-in scratch for the allocation-free entry point -----------------------------------------
+// Status block + per-row partial statistics for up to kStaticMaxTiles output tiles (4 MiB + 256 B).
+// Every device that loads this library carries the array until the process exits.  In host code
+// the name below is only a handle for cudaGetSymbolAddress; kernels receive the device address.
+constexpr size_t kStaticMaxTiles = 2048;
+constexpr size_t kStaticScratchBytes = kStatusBytes + kStaticMaxTiles * BM * sizeof(float4);
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+size_t tc_static_scratch_bytes() { return kStaticScratchBytes; }
+
+kf_status tc_static_scratch(void** ptr) {
+    static std::mutex mu;
+    static void* cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return KF_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!cached[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return KF_ERR_CUDA;
+        cached[dev] = p;
+    }
+    *ptr = cached[dev];
+    return KF_OK;
+}
+
 static cudaEvent_t g_split_event = nullptr;
 void tc_set_split_event(cudaEvent_t ev) { g_split_event = ev; }
 

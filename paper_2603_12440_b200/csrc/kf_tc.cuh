@@ -15,6 +15,11 @@ kf_status launch_tc_linear(const void* X, long long ldx, const void* W, long lon
                            long long M, long long N, long long K, const EpilogueParams& ep, const RowNormParams& rn,
                            void* ws, int grid_override, cudaStream_t st, int* grid_out);
 
+// scratch built into the library image (allocation-free entry point): device address for the current
+// device, resolved once per device, and its size
+kf_status tc_static_scratch(void** ptr);
+size_t tc_static_scratch_bytes();
+
 // profiling aid: event recorded between the GEMM kernel and the finishing kernel (nullptr = off)
 void tc_set_split_event(cudaEvent_t ev);
 

@@ -1,0 +1,77 @@
+"""The allocation-free entry point, kf_linear_epilogue_rownorm_noalloc.
+
+Some users of this library are handed their input and output buffers and nothing else: a plug-in
+inside an application whose memory pool is off limits, or a service where cudaMalloc after start-up
+is banned because it stalls the device and may fail.  They cannot supply the scratch buffer the
+normal call wants, so this form keeps its scratch (status block + per-row partial statistics) in an
+array built into the library.  The tests drive it through the C ABI and hold it to the output of
+the normal entry point -- same kernels, so the results must be identical -- on two calls in a row
+that reuse the shared array with different shapes and row ops.
+
+Collected last on purpose (file name), so a failure here cannot hide the other tests' results.
+"""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2603_12440_b200 import inputs
+from tests.helpers import assert_parity, oracle_of, problem_to_device, to_f64
+
+
+@pytest.fixture(scope="module")
+def kf():
+    import paper_2603_12440_b200 as m
+    m.binding.lib()
+    return m
+
+
+def _problem(seed, M, N, K, norm, act):
+    return inputs.make_problem(f"noalloc{seed}", "bf16", M, N, K, seed=seed, std_x=1.0, std_w=1.0 / np.sqrt(K),
+                               bias_std=0.5, residual_std=1.0,
+                               gamma_std=0.1 if norm in ("layernorm", "rmsnorm") else None,
+                               beta_std=0.1 if norm == "layernorm" else None, act=act, norm=norm)
+
+
+@pytest.mark.gpu
+def test_noalloc_matches_the_workspace_entry_point_twice_in_a_row(kf):
+    # first call: 3 x 9 tiles, softmax; second call: 2 x 3 tiles, LayerNorm -- the second reuses the
+    # array the first one filled, with a different tile grid and a different meaning of the partials
+    cases = [_problem(71, 300, 2056, 200, "softmax", "gelu_erf"), _problem(72, 200, 520, 136, "layernorm", "silu")]
+    for p in cases:
+        d = problem_to_device(p)
+        assert kf.tile_config(p.M, p.N, p.K, torch.bfloat16, p.norm)["kernel"] == 3
+        want = kf.linear_epilogue_rownorm(d["X"], d["W"], d["bias"], p.act, p.scale, d["residual"], p.norm,
+                                          d["gamma"], d["beta"], p.eps)
+        kf.check_device_status()
+        out = torch.full((p.M, p.N), float("nan"), dtype=torch.bfloat16, device="cuda")
+        got = kf.linear_epilogue_rownorm_noalloc(d["X"], d["W"], out, d["bias"], p.act, p.scale, d["residual"],
+                                                 p.norm, d["gamma"], d["beta"], p.eps, wait=True)
+        assert got.data_ptr() == out.data_ptr()
+        assert torch.equal(got, want), "same kernels on the same inputs must give the same bits"
+        assert_parity(to_f64(got), oracle_of(p), "bf16", f"noalloc {p.norm}")
+    # asynchronous form (no status read-back), same stream: still ordered after the calls above
+    p = cases[0]
+    d = problem_to_device(p)
+    out = torch.empty((p.M, p.N), dtype=torch.bfloat16, device="cuda")
+    kf.linear_epilogue_rownorm_noalloc(d["X"], d["W"], out, d["bias"], p.act, p.scale, d["residual"], p.norm)
+    torch.cuda.synchronize()
+    assert_parity(to_f64(out), oracle_of(p), "bf16", "noalloc async")
+
+
+def test_noalloc_rejects_problems_beyond_its_scratch(kf):
+    # host-side check: nothing is launched, so this runs without a GPU (pointers are never touched)
+    b = kf.binding
+    L = b.lib()
+    P = 0x10000000
+    ep = b._Epilogue(None, 0, 1.0, None, 0)
+    rn = b._RowNorm(1, None, None, 0.0)
+    M, N, K = 128 * 2049, 256, 64                     # 2049 output tiles > 2048
+    st = L.kf_linear_epilogue_rownorm_noalloc(P, K, P, K, P, N, M, N, K, 1, ctypes.byref(ep), ctypes.byref(rn), None, None)
+    assert st == 7 and kf.status_string(7) == "KF_ERR_SCRATCH_LIMIT"
+    # without a row-norm only the status block is needed: the size check lets the call through to the
+    # ordinary validation (here: a null output pointer)
+    rn0 = b._RowNorm(0, None, None, 0.0)
+    st = L.kf_linear_epilogue_rownorm_noalloc(P, K, P, K, None, N, 0, N, K, 1, ctypes.byref(ep), ctypes.byref(rn0), None, None)
+    assert st == 0                                    # M == 0: nothing to do
