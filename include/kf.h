@@ -94,7 +94,7 @@ typedef struct {
  * the best-measured instantiation of a templated kernel is the one that is used). */
 typedef struct {
     int32_t kernel;           /* 0 none, 1 SIMT row-resident, 2 SIMT tiled, 3 tcgen05 */
-    int32_t bm, bn, bk;       /* CTA tile */
+    int32_t bm, bn, bk;       /* tile of one work unit (a CTA, or a CTA pair when cta_group is 2) */
     int32_t stages;           /* shared-memory pipeline depth */
     int32_t cta_group;        /* 1 or 2 CTAs per MMA */
     int32_t epilogue_warps;
@@ -163,11 +163,11 @@ size_t kf_host_call_bytes(int64_t M, int64_t N, int64_t K, kf_dtype dt, int has_
  * array compiled into the library's device image.
  *
  * Same arguments, results and kernels as kf_linear_epilogue_rownorm, minus ws / ws_bytes.
- *   - Limit: kf_workspace_bytes(M,N,K,dt,norm) must not exceed 4 MiB + 256 bytes, i.e. a bf16
+ *   - Limit: kf_workspace_bytes(M,N,K,dt,norm) must not exceed 8 MiB + 256 bytes, i.e. a bf16
  *     row-norm may span at most 2048 output tiles of 128 x 256 (ceil(M/128) * ceil(N/256)).  Larger
  *     problems return KF_ERR_SCRATCH_LIMIT and launch nothing.  Calls without a row-norm and fp32
  *     calls need only the status block and are never rejected for size.
- *   - Every device that loads the library holds the 4 MiB array until the process exits.
+ *   - Every device that loads the library holds the 8 MiB array until the process exits.
  *   - The call performs no cudaMalloc / cudaFree and calls no allocating routine.  The first call
  *     on each device looks the array's device address up (cudaGetSymbolAddress, with that device
  *     current, which may load the module); make that first call before starting any stream capture.
@@ -198,7 +198,7 @@ kf_status kf_check_device_status(void *ws, void *stream, uint32_t *detail);
 
 /* Step a7: resolve a call to its kernel and tile shape without launching anything.  `aligned`
  * says whether all pointers and pitches of the call will be 16-byte aligned.  The environment
- * variable KF_TILE_OVERRIDE="stages=S,epi=E,grid=G,scheme=R,kernel=Q" overrides table fields
+ * variable KF_TILE_OVERRIDE="kernel=Q,cg=C,grid=G" overrides the kernel family, CTAs per MMA and grid
  * (for sweeps). */
 kf_status kf_tile_config_query(int64_t M, int64_t N, int64_t K, kf_dtype dt, kf_norm norm,
                                int aligned, kf_tile_config *out);

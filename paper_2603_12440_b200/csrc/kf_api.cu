@@ -15,7 +15,7 @@ inline bool is_aligned(const void* p, size_t a) { return (reinterpret_cast<uintp
 inline size_t round256(size_t b) { return (b + 255) & ~(size_t)255; }
 
 struct Override {
-    int kernel = 0, grid = 0;
+    int kernel = 0, grid = 0, cg = 0;
 };
 const Override& env_override() {
     static Override o = [] {
@@ -25,6 +25,7 @@ const Override& env_override() {
         const char* p;
         if ((p = std::strstr(e, "kernel="))) v.kernel = std::atoi(p + 7);
         if ((p = std::strstr(e, "grid="))) v.grid = std::atoi(p + 5);
+        if ((p = std::strstr(e, "cg="))) v.cg = std::atoi(p + 3);
         return v;
     }();
     return o;
@@ -44,11 +45,12 @@ kf_status resolve(long long M, long long N, long long K, int dt, int norm, bool 
         use_tc = false;
     if (use_tc) {
         c->kernel = 3;
-        tc_tile_shape(&c->bm, &c->bn, &c->bk, &c->stages, &c->epilogue_warps);
-        c->cta_group = 1;
+        c->cta_group = (ov.cg == 1 || ov.cg == 2) ? ov.cg : tc_default_cta_group(M, N);
+        tc_tile_shape(c->cta_group, &c->bm, &c->bn, &c->bk, &c->stages, &c->epilogue_warps);
         c->row_scheme = norm == KF_NORM_NONE ? 0 : 2;
-        c->grid = tc_default_grid(M, N);
-        if (ov.grid > 0 && ov.grid < c->grid) c->grid = ov.grid;
+        c->grid = tc_default_grid(M, N, c->cta_group);
+        if (ov.grid > 0 && ov.grid < c->grid) c->grid = ov.grid - ov.grid % c->cta_group;
+        if (c->grid < c->cta_group) c->grid = c->cta_group;
         return KF_OK;
     }
     bool rows = simt_row_resident_ok(N) && (norm != KF_NORM_NONE ? (M < 4096 || dt == KF_BF16) : (M <= 1024));
@@ -117,7 +119,7 @@ kf_status linear_impl(const void* X, int64_t ldx, const void* W, int64_t ldw, vo
     if (cfg.kernel == 3) {
         const size_t need = kStatusBytes + (rn.norm != KF_NORM_NONE ? tc_partials_bytes(M, N) : 0);
         if (!ws || ws_bytes < need) return KF_ERR_WORKSPACE;
-        return launch_tc_linear(X, ldx, W, ldw, Y, ldy, M, N, K, ep, rn, ws, env_override().grid, st, nullptr);
+        return launch_tc_linear(X, ldx, W, ldw, Y, ldy, M, N, K, ep, rn, ws, cfg.cta_group, env_override().grid, st, nullptr);
     }
     cudaError_t e = launch_simt_linear(X, ldx, W, ldw, Y, ldy, M, N, K, dt, ep, rn, cfg.kernel == 1, st, nullptr);
     return e == cudaSuccess ? KF_OK : KF_ERR_CUDA;

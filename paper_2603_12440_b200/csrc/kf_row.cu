@@ -131,6 +131,204 @@ row_norm_reg_kernel(const T* X, long long ldx, T* Y, long long ldy, long long M,
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Ring kernel: persistent CTAs, one producer thread streaming whole rows into a shared-memory ring
+// with bulk async copies (cp.async.bulk + mbarrier), and consumer warps that each take a row of the
+// ring, sweep it twice out of shared memory (moments about a shift, then the output), reduce with
+// shuffles and store the normalised row with streaming 128-bit stores.  The bytes in flight per SM
+// are set by the ring (up to ~190 KiB), not by occupancy, and no thread waits on a global load.
+#ifndef KF_RING_CONSUMERS
+#define KF_RING_CONSUMERS 16
+#endif
+constexpr int kRingConsumers = KF_RING_CONSUMERS;
+constexpr int kRingThreads = 32 * (kRingConsumers + 1);
+constexpr long long kRingTimeoutCycles = 3000000000ll;
+
+__device__ unsigned int g_row_ring_status = 0;      // set to 1 if a bounded wait ever gave up
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void rbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void rbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void rbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// bounded wait; false = gave up (recorded), the caller abandons its remaining rows
+__device__ __forceinline__ bool rbar_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok = 0, spins = 0;
+    long long t0 = 0;
+    for (;;) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (ok) return true;
+        if (spins == 0) t0 = clock64();
+        if ((++spins & 0xFF) == 0 && clock64() - t0 > kRingTimeoutCycles) {
+            atomicExch(&g_row_ring_status, 1u);
+            return false;
+        }
+    }
+}
+__device__ __forceinline__ void bulk_load_row(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+
+template <typename T, int NORM, int VPT>
+__global__ void __launch_bounds__(kRingThreads, 1)
+row_norm_ring_kernel(const T* X, long long ldx, T* Y, long long ldy, long long M, int N, int slots,
+                     const T* __restrict__ gamma, const T* __restrict__ beta, float eps) {
+    constexpr int E = Elem<T>::kVec;
+    extern __shared__ __align__(128) uint8_t ring_smem[];
+    const int NV = N / E;
+    const uint32_t row_bytes = (uint32_t)N * sizeof(T);
+    // layout: [slots x row_bytes][gamma lo/hi float4 arrays][beta lo/hi float4 arrays][barriers]
+    uint8_t* ring = ring_smem;
+    float4* gam = reinterpret_cast<float4*>(ring_smem + (size_t)slots * row_bytes);
+    float4* bet = gam + (NORM == KF_NORM_SOFTMAX ? 0 : (E / 4) * NV);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(bet + (NORM == KF_NORM_LAYERNORM ? (E / 4) * NV : 0));
+    const uint32_t bar0 = smem_addr(bars);
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (slots + s); };
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < slots; ++s) {
+            rbar_init(full_bar(s), 1);
+            rbar_init(empty_bar(s), 1);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // gamma / beta as fp32, de-interleaved so that a lane's two float4 halves are conflict-free reads
+    if (NORM != KF_NORM_SOFTMAX) {
+        for (int idx = threadIdx.x; idx < NV; idx += kRingThreads) {
+            float g[E], b[E];
+#pragma unroll
+            for (int e = 0; e < E; ++e) { g[e] = 1.f; b[e] = 0.f; }
+            if (gamma) unpack<T>(__ldg(reinterpret_cast<const uint4*>(gamma) + idx), g);
+            if (beta && NORM == KF_NORM_LAYERNORM) unpack<T>(__ldg(reinterpret_cast<const uint4*>(beta) + idx), b);
+#pragma unroll
+            for (int h = 0; h < E / 4; ++h) {
+                gam[h * NV + idx] = make_float4(g[h * 4], g[h * 4 + 1], g[h * 4 + 2], g[h * 4 + 3]);
+                if (NORM == KF_NORM_LAYERNORM)
+                    bet[h * NV + idx] = make_float4(b[h * 4], b[h * 4 + 1], b[h * 4 + 2], b[h * 4 + 3]);
+            }
+        }
+    }
+    __syncthreads();
+
+    // rows of this CTA: blockIdx.x, blockIdx.x + gridDim.x, ...; its i-th row uses slot i % slots
+    const long long my_rows = (M - blockIdx.x + gridDim.x - 1) / gridDim.x;
+
+    if (warp == kRingConsumers) {
+        if (lane == 0) {
+            for (long long i = 0; i < my_rows; ++i) {
+                const int s = (int)(i % slots);
+                const uint32_t ph = (uint32_t)((i / slots) & 1);
+                if (!rbar_wait(empty_bar(s), ph ^ 1u)) break;
+                rbar_expect_tx(full_bar(s), row_bytes);
+                const long long row = blockIdx.x + i * (long long)gridDim.x;
+                bulk_load_row(smem_addr(ring + (size_t)s * row_bytes), X + row * ldx, row_bytes, full_bar(s));
+            }
+        }
+        return;
+    }
+
+    for (long long i = warp; i < my_rows; i += kRingConsumers) {
+        const int s = (int)(i % slots);
+        const uint32_t ph = (uint32_t)((i / slots) & 1);
+        const long long row = blockIdx.x + i * (long long)gridDim.x;
+        if (!rbar_wait(full_bar(s), ph)) break;
+        const uint4* srow = reinterpret_cast<const uint4*>(ring + (size_t)s * row_bytes);
+        uint4* yr = reinterpret_cast<uint4*>(Y + row * ldy);
+        // The row stays in shared memory and is swept twice (statistics, then output), so a warp needs
+        // few registers and many warps fit: latency is hidden by warps, not by a register-resident row.
+        float x[E];
+        if (NORM == KF_NORM_SOFTMAX) {
+            float m[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+            for (int v = 0; v < VPT; ++v)
+                if (lane + v * 32 < NV) {
+                    unpack<T>(srow[lane + v * 32], x);
+#pragma unroll
+                    for (int e = 0; e < E; ++e) m[e & 3] = fmaxf(m[e & 3], x[e]);
+                }
+            const float ms = warp_max(fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3]))) * kLog2e;
+            float l[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int v = 0; v < VPT; ++v)
+                if (lane + v * 32 < NV) {
+                    unpack<T>(srow[lane + v * 32], x);
+#pragma unroll
+                    for (int e = 0; e < E; ++e) l[e & 3] += exp2f(fmaf(x[e], kLog2e, -ms));
+                }
+            const float inv = 1.0f / warp_sum((l[0] + l[1]) + (l[2] + l[3]));
+#pragma unroll
+            for (int v = 0; v < VPT; ++v) {
+                const int idx = lane + v * 32;
+                if (idx < NV) {
+                    unpack<T>(srow[idx], x);
+#pragma unroll
+                    for (int e = 0; e < E; ++e) x[e] = exp2f(fmaf(x[e], kLog2e, -ms)) * inv;
+                    st_stream(yr + idx, pack<T>(x));
+                }
+            }
+        } else {
+            // one sweep for both moments about a shift taken from the row itself (its first element):
+            // sum(x - c) and sum((x - c)^2) lose no accuracy to cancellation because c lies inside the data
+            const float c = (NORM == KF_NORM_LAYERNORM) ? Elem<T>::load(reinterpret_cast<const T*>(srow)) : 0.f;
+            float a[4] = {0.f, 0.f, 0.f, 0.f}, q[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int v = 0; v < VPT; ++v)
+                if (lane + v * 32 < NV) {
+                    unpack<T>(srow[lane + v * 32], x);
+#pragma unroll
+                    for (int e = 0; e < E; ++e) {
+                        const float d = x[e] - c;
+                        a[e & 3] += d;
+                        q[e & 3] = fmaf(d, d, q[e & 3]);
+                    }
+                }
+            const float s1 = warp_sum((a[0] + a[1]) + (a[2] + a[3]));
+            const float s2 = warp_sum((q[0] + q[1]) + (q[2] + q[3]));
+            const float dm = (NORM == KF_NORM_LAYERNORM) ? s1 / (float)N : 0.f;      // mean - c
+            const float var = fmaxf(s2 / (float)N - dm * dm, 0.f);
+            const float rstd = rsqrtf(var + eps);
+            const float shift = c + dm;                                              // the mean (0 for RMSNorm)
+#pragma unroll
+            for (int v = 0; v < VPT; ++v) {
+                const int idx = lane + v * 32;
+                if (idx < NV) {
+                    unpack<T>(srow[idx], x);
+#pragma unroll
+                    for (int h = 0; h < E / 4; ++h) {
+                        const float4 g = gam[h * NV + idx];
+                        float* o = &x[h * 4];
+                        if (NORM == KF_NORM_LAYERNORM) {
+                            const float4 b = bet[h * NV + idx];
+                            o[0] = fmaf((o[0] - shift) * rstd, g.x, b.x); o[1] = fmaf((o[1] - shift) * rstd, g.y, b.y);
+                            o[2] = fmaf((o[2] - shift) * rstd, g.z, b.z); o[3] = fmaf((o[3] - shift) * rstd, g.w, b.w);
+                        } else {
+                            o[0] *= rstd * g.x; o[1] *= rstd * g.y; o[2] *= rstd * g.z; o[3] *= rstd * g.w;
+                        }
+                    }
+                    st_stream(yr + idx, pack<T>(x));
+                }
+            }
+        }
+        __syncwarp();
+        if (lane == 0) rbar_arrive(empty_bar(s));           // every lane has finished reading the slot
+    }
+}
+
 // generic: one CTA per row, scalar accesses, any N / alignment; Y may alias X
 template <typename T, int NORM>
 __global__ void __launch_bounds__(kRowThreads)
@@ -194,13 +392,69 @@ cudaError_t launch_typed(const void* X, long long ldx, void* Y, long long ldy, l
         }
         return cudaGetLastError();
     }
-    // threads per row / vectors per thread: one warp per row while a row fits 16 vectors a lane
-    int tpr = 32;
-    if (NV > 32 * 16) { tpr = 64; while (tpr < 512 && (long long)tpr * 8 < NV) tpr <<= 1; }
-    static const int env_tpr = [] {                              // sweep hook, read once
+    static const int env_tpr = [] {                              // sweep hooks, read once
         const char* e = std::getenv("KF_ROW_TPR");
         return e ? std::atoi(e) : 0;
     }();
+    static const int env_ring = [] {
+        const char* e = std::getenv("KF_ROW_RING");
+        return e ? std::atoi(e) : -1;
+    }();
+    static const int sms = [] {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) return 148;
+        return v;
+    }();
+    // ring kernel: a row fits one warp's registers, rows start 16-byte aligned, Y does not alias X
+    // (the producer runs ahead of the stores), and there are enough rows to fill persistent CTAs
+    const bool ring_ok = NV <= 32 * 16 && (const void*)X != (const void*)Y && M >= 4ll * sms && env_tpr == 0 &&
+                         env_ring != 0;
+    if (ring_ok) {
+        const int need_v = (int)((NV + 31) / 32);
+        int vpt = 1;
+        while (vpt < need_v) vpt <<= 1;
+        const size_t row_bytes = (size_t)N * sizeof(T);
+        const size_t vec_bytes = (NORM == KF_NORM_SOFTMAX ? 0 : (NORM == KF_NORM_LAYERNORM ? 2 : 1)) * (size_t)N * 4;
+        const size_t budget = 226 * 1024;
+        long long slots = ((long long)budget - (long long)vec_bytes - 64) / (long long)(row_bytes + 16);
+        // a slot must always come back to the same consumer warp (row i -> slot i % slots, warp
+        // i % consumers): then a warp only ever waits for the phase right after one it consumed itself
+        slots -= slots % kRingConsumers;
+        if (slots > 4 * kRingConsumers) slots = 4 * kRingConsumers;
+        if (slots >= kRingConsumers) {
+            const size_t smem = slots * row_bytes + vec_bytes + 2 * slots * 8;
+            const int grid = (int)(M < sms ? M : sms);
+            cudaError_t e = cudaSuccess;
+#define KF_RING_LAUNCH(V)                                                                                      \
+    do {                                                                                                       \
+        static bool attr_done[64] = {};                                                                        \
+        int dev = 0;                                                                                           \
+        cudaGetDevice(&dev);                                                                                   \
+        if (dev >= 0 && dev < 64 && !attr_done[dev]) {                                                         \
+            e = cudaFuncSetAttribute(row_norm_ring_kernel<T, NORM, V>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                     226 * 1024);                                                              \
+            attr_done[dev] = e == cudaSuccess;                                                                 \
+        }                                                                                                      \
+        if (e == cudaSuccess)                                                                                  \
+            row_norm_ring_kernel<T, NORM, V><<<grid, kRingThreads, smem, st>>>(x, ldx, y, ldy, M, (int)N,      \
+                                                                               (int)slots, g, b, rn.eps);      \
+    } while (0)
+            switch (vpt) {
+            case 1: KF_RING_LAUNCH(1); break;
+            case 2: KF_RING_LAUNCH(2); break;
+            case 4: KF_RING_LAUNCH(4); break;
+            case 8: KF_RING_LAUNCH(8); break;
+            default: KF_RING_LAUNCH(16); break;
+            }
+#undef KF_RING_LAUNCH
+            if (e != cudaSuccess) return e;
+            return cudaGetLastError();
+        }
+    }
+    // threads per row / vectors per thread: one warp per row while a row fits 16 vectors a lane
+    int tpr = 32;
+    if (NV > 32 * 16) { tpr = 64; while (tpr < 512 && (long long)tpr * 8 < NV) tpr <<= 1; }
     if (env_tpr >= 32 && env_tpr <= 512 && (env_tpr & (env_tpr - 1)) == 0 && (long long)env_tpr * 16 >= NV)
         tpr = env_tpr;
     const int need = (int)((NV + tpr - 1) / tpr);

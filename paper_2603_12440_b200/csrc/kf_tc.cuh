@@ -5,15 +5,17 @@
 namespace kf {
 
 // tile shape the tensor-core kernel was built with
-void tc_tile_shape(int* bm, int* bn, int* bk, int* stages, int* epi_warps);
+void tc_tile_shape(int cta_group, int* bm, int* bn, int* bk, int* stages, int* epi_warps);
+// 1 or 2 CTAs per MMA for this shape (2 = CTA pairs sharing the W tile)
+int tc_default_cta_group(long long M, long long N);
 // bytes of per-row, per-tile partial statistics behind the status block of the workspace
 size_t tc_partials_bytes(long long M, long long N);
-int tc_default_grid(long long M, long long N);
+int tc_default_grid(long long M, long long N, int cta_group);
 // launches the persistent GEMM (+ finishing kernel for a row-norm); all pointers 16-byte aligned,
 // K, N and every pitch multiples of 8, K >= 1
 kf_status launch_tc_linear(const void* X, long long ldx, const void* W, long long ldw, void* Y, long long ldy,
                            long long M, long long N, long long K, const EpilogueParams& ep, const RowNormParams& rn,
-                           void* ws, int grid_override, cudaStream_t st, int* grid_out);
+                           void* ws, int cta_group, int grid_override, cudaStream_t st, int* grid_out);
 
 // scratch built into the library image (allocation-free entry point): device address for the current
 // device, resolved once per device, and its size

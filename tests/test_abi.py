@@ -44,10 +44,10 @@ def test_workspace_bytes(kf):
     import torch
     assert kf.workspace_bytes(128, 256, 256, torch.float32, "softmax") == 256
     assert kf.workspace_bytes(8192, 4096, 4096, torch.bfloat16, "none") == 256
-    # bf16 row-norm: one float4 per row per 256-column tile, rows padded to 128, after the status block
-    assert kf.workspace_bytes(4096, 8192, 2048, torch.bfloat16, "layernorm") == 256 + 32 * 32 * 128 * 16
-    assert kf.workspace_bytes(2048, 32768, 1024, torch.bfloat16, "softmax") == 256 + 16 * 128 * 128 * 16
-    assert kf.workspace_bytes(100, 300, 64, torch.bfloat16, "rmsnorm") == 256 + 1 * 2 * 128 * 16
+    # bf16 row-norm: one float4 per row per 128-column sub-tile, rows padded to 128, after the status block
+    assert kf.workspace_bytes(4096, 8192, 2048, torch.bfloat16, "layernorm") == 256 + 4096 * 64 * 16
+    assert kf.workspace_bytes(2048, 32768, 1024, torch.bfloat16, "softmax") == 256 + 2048 * 256 * 16
+    assert kf.workspace_bytes(100, 300, 64, torch.bfloat16, "rmsnorm") == 256 + 128 * 3 * 16
 
 
 def test_tile_table_on_the_five_configs(kf):
@@ -55,8 +55,12 @@ def test_tile_table_on_the_five_configs(kf):
     c1 = kf.tile_config(128, 256, 256, torch.float32, "softmax")
     assert c1["kernel"] == 1 and c1["row_scheme"] == 1            # fp32: CUDA cores, rows resident in a CTA
     c3 = kf.tile_config(8192, 4096, 4096, torch.bfloat16, "none")
-    assert (c3["kernel"], c3["bm"], c3["bn"], c3["bk"], c3["row_scheme"]) == (3, 128, 256, 64, 0)
-    assert 1 <= c3["grid"] <= 1024
+    # large bf16: CTA pairs (cta_group 2) computing 256 x 256 per work unit from a 7-stage ring
+    assert (c3["kernel"], c3["bm"], c3["bn"], c3["bk"], c3["cta_group"], c3["stages"], c3["row_scheme"]) == \
+        (3, 256, 256, 64, 2, 7, 0)
+    assert 2 <= c3["grid"] <= 1024 and c3["grid"] % 2 == 0
+    one_block = kf.tile_config(128, 4096, 4096, torch.bfloat16, "none")      # a single row block cannot pair up
+    assert (one_block["cta_group"], one_block["bm"], one_block["stages"]) == (1, 128, 4)
     c4 = kf.tile_config(4096, 8192, 2048, torch.bfloat16, "layernorm")
     assert c4["kernel"] == 3 and c4["row_scheme"] == 2
     c5 = kf.tile_config(2048, 32768, 1024, torch.bfloat16, "softmax")

@@ -44,6 +44,28 @@ def test_row_ops_match_oracle(kf, dtype, M, N):
     torch.cuda.synchronize()
 
 
+# enough rows for the persistent ring kernel (bulk-copy producer + register consumers): row lengths
+# from one vector per lane to the 16-vector maximum, ragged vector counts, ring wrap-around
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("M,N", [(700, 64), (1500, 1000), (2500, 2048), (5000, 4096), (3001, 3080)])
+def test_row_ops_ring_kernel(kf, dtype, M, N):
+    if dtype == "f32" and N > 2048:
+        N //= 2                                     # one warp holds at most 8 KiB of a row
+    X, g, b = _draw(200 + N, M, N, dtype, std=1.5, shift=-0.25)
+    dX, dg, db = to_device(X, dtype), to_device(g, dtype), to_device(b, dtype)
+    assert_parity(to_f64(kf.row_layernorm(dX, dg, db, 1e-5)), kfo.row_layernorm(X, g, b, 1e-5), dtype, f"ring ln {M}x{N}")
+    assert_parity(to_f64(kf.row_softmax(dX)), kfo.row_softmax(X), dtype, f"ring softmax {M}x{N}")
+    assert_parity(to_f64(kf.row_rmsnorm(dX, dg, 1e-6)), kfo.row_rmsnorm(X, g, 1e-6), dtype, f"ring rms {M}x{N}")
+    assert_parity(to_f64(kf.row_layernorm(dX, None, None, 1e-5)), kfo.row_layernorm(X, None, None, 1e-5), dtype, "ring ln plain")
+    # padded pitches on both sides, canary columns untouched
+    big = torch.full((M, N + 16), 3.0, dtype=dX.dtype, device="cuda")
+    big[:, :N] = dX
+    out = torch.full((M, N + 8), 5.0, dtype=dX.dtype, device="cuda")
+    kf.row_layernorm(big[:, :N], dg, db, 1e-5, out=out[:, :N])
+    assert_parity(to_f64(out[:, :N]), kfo.row_layernorm(X, g, b, 1e-5), dtype, "ring ln padded")
+    assert bool((out[:, N:] == 5.0).all())
+
+
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
 def test_row_ops_in_place_padded_pitch_and_unaligned(kf, dtype):
     M, N = 50, 2048
