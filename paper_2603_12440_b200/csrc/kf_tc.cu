@@ -279,6 +279,15 @@ struct TcParams {
 // 8-column vectors at or beyond N are not read from the residual.
 __device__ __forceinline__ void epilogue32(float (&a)[32], const TcParams& p, const float* bias32, long long row,
                                            int col0, bool row_ok) {
+    // the residual comes from global memory (often DRAM): issue its loads first, use them last
+    const bool has_res = p.residual && row_ok && !(p.debug & 64);
+    uint4 rv[4];
+    if (has_res) {
+        const int left = p.N - col0;
+        const uint4* rp = reinterpret_cast<const uint4*>(p.residual + row * p.ldr + col0);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) rv[q] = (q * 8 < left) ? __ldg(rp + q) : make_uint4(0, 0, 0, 0);
+    }
     if (bias32) {
         const float4* bp = reinterpret_cast<const float4*>(bias32);
 #pragma unroll
@@ -315,12 +324,7 @@ __device__ __forceinline__ void epilogue32(float (&a)[32], const TcParams& p, co
 #pragma unroll
         for (int e = 0; e < 32; ++e) a[e] *= p.scale;
     }
-    if (p.residual && row_ok && !(p.debug & 64)) {
-        const int left = p.N - col0;
-        const uint4* rp = reinterpret_cast<const uint4*>(p.residual + row * p.ldr + col0);
-        uint4 rv[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) rv[q] = (q * 8 < left) ? __ldg(rp + q) : make_uint4(0, 0, 0, 0);
+    if (has_res) {
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
             float r[8];
@@ -638,44 +642,63 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
 }
 
 // ------------------------------------------------------------------------------ finishing kernel
-// One warp per row: merge the row's per-sub-tile partials with warp shuffles, then rescale the 16-bit
-// intermediates of the row in place (128-bit accesses, several in flight per lane).
+// WPR warps per row (1, 2, 4 or 8; a CTA of 8 warps holds 8 / WPR rows): merge the row's per-sub-tile
+// partials (warp shuffles + one shared-memory hop across the row's warps), then rescale the 16-bit
+// intermediates of the row in place with up to 8 independent 128-bit accesses in flight per lane.
 constexpr int kFinWarps = 8;
 
+template <bool IS_MAX>
+__device__ __forceinline__ float fin_group_reduce(float v, int wpr, int warp, float* red) {
+    v = IS_MAX ? warp_max(v) : warp_sum(v);
+    if (wpr == 1) return v;
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) red[warp] = v;
+    __syncthreads();
+    const int g0 = (warp / wpr) * wpr;
+    float t = red[g0];
+    for (int i = 1; i < wpr; ++i) t = IS_MAX ? fmaxf(t, red[g0 + i]) : t + red[g0 + i];
+    return t;
+}
+
 __global__ void __launch_bounds__(kFinWarps * 32)
-tc_rownorm_finish_kernel(__nv_bfloat16* Y, long long ldy, int M, int N, int nsub, const float4* __restrict__ partials,
-                         int norm, const __nv_bfloat16* __restrict__ gamma, const __nv_bfloat16* __restrict__ beta,
-                         float eps) {
-    extern __shared__ float2 coef_smem[];               // per warp: nsub x {multiplier, offset}
+tc_rownorm_finish_kernel(__nv_bfloat16* Y, long long ldy, int M, int N, int nsub, int wpr,
+                         const float4* __restrict__ partials, int norm, const __nv_bfloat16* __restrict__ gamma,
+                         const __nv_bfloat16* __restrict__ beta, float eps) {
+    extern __shared__ float2 coef_smem[];               // per row of the CTA: nsub x {multiplier, offset}
+    __shared__ float red[kFinWarps];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const long long row = (long long)blockIdx.x * kFinWarps + warp;
-    if (row >= M) return;
-    float2* coef = coef_smem + (size_t)warp * nsub;
+    const int rows_per_cta = kFinWarps / wpr;
+    const int grow = warp / wpr;                         // row of this CTA
+    const int gt = (warp % wpr) * 32 + lane, gsize = wpr * 32;     // thread index / count within the row's group
+    long long row = (long long)blockIdx.x * rows_per_cta + grow;
+    const bool live = row < M;
+    if (!live) row = M - 1;                              // keep every thread in the barriers; stores are skipped
+    float2* coef = coef_smem + (size_t)grow * nsub;
     const float4* pr = partials + (size_t)row * nsub;   // rows of a padded row block are contiguous
     float rstd = 1.f;
 
     if (norm == KF_NORM_SOFTMAX) {
         float m = -INFINITY;
-        for (int s = lane; s < nsub; s += 32) m = fmaxf(m, pr[s].x);
-        m = warp_max(m);
+        for (int s = gt; s < nsub; s += gsize) m = fmaxf(m, pr[s].x);
+        m = fin_group_reduce<true>(m, wpr, warp, red);
         float l = 0.f;
-        for (int s = lane; s < nsub; s += 32) {
+        for (int s = gt; s < nsub; s += gsize) {
             const float4 q = pr[s];
             const float f = exp2f((q.x - m) * kLog2e);
             coef[s] = make_float2(f, 0.f);
             l = fmaf(q.y, f, l);
         }
-        rstd = 1.0f / warp_sum(l);
+        rstd = 1.0f / fin_group_reduce<false>(l, wpr, warp, red);
     } else if (norm == KF_NORM_LAYERNORM) {
         float sum = 0.f;
-        for (int s = lane; s < nsub; s += 32) {
+        for (int s = gt; s < nsub; s += gsize) {
             const float4 q = pr[s];
             const float cnt = (float)min(kSub, N - s * kSub);
             sum += q.x * cnt + q.y;               // sum of a over the sub-tile = shift * count + sum(a - shift)
         }
-        const float mean = warp_sum(sum) / (float)N;
+        const float mean = fin_group_reduce<false>(sum, wpr, warp, red) / (float)N;
         float m2 = 0.f;
-        for (int s = lane; s < nsub; s += 32) {
+        for (int s = gt; s < nsub; s += gsize) {
             const float4 q = pr[s];
             const float cnt = (float)min(kSub, N - s * kSub);
             const float dmean = q.y / cnt;                       // sub-tile mean minus its shift
@@ -684,33 +707,34 @@ tc_rownorm_finish_kernel(__nv_bfloat16* Y, long long ldy, int M, int N, int nsub
             m2 += fmaf(cnt * d, d, m2_t);                        // Chan's merge
             coef[s] = make_float2(q.w, q.x - mean);
         }
-        rstd = rsqrtf(warp_sum(m2) / (float)N + eps);
+        rstd = rsqrtf(fin_group_reduce<false>(m2, wpr, warp, red) / (float)N + eps);
     } else {
         float ss = 0.f;
-        for (int s = lane; s < nsub; s += 32) {
+        for (int s = gt; s < nsub; s += gsize) {
             const float4 q = pr[s];
             ss += q.z;
             coef[s] = make_float2(q.w, 0.f);
         }
-        rstd = rsqrtf(warp_sum(ss) / (float)N + eps);
+        rstd = rsqrtf(fin_group_reduce<false>(ss, wpr, warp, red) / (float)N + eps);
     }
-    __syncwarp();
+    __syncthreads();                                     // coef of the row is complete
+    if (!live) return;
 
     uint4* yr = reinterpret_cast<uint4*>(Y + row * ldy);
     const uint4* gv = reinterpret_cast<const uint4*>(gamma);
     const uint4* bv = reinterpret_cast<const uint4*>(beta);
     const int NV = N / 8;
     constexpr int U = 4;                                 // vectors in flight per lane
-    for (int i0 = lane; i0 < NV; i0 += 32 * U) {
+    for (int i0 = gt; i0 < NV; i0 += gsize * U) {
         uint4 raw[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const int idx = i0 + u * 32;
+            const int idx = i0 + u * gsize;
             if (idx < NV) raw[u] = yr[idx];
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const int idx = i0 + u * 32;
+            const int idx = i0 + u * gsize;
             if (idx >= NV) break;
             float f[8];
             const float2 c = coef[idx / (kSub / 8)];
@@ -881,8 +905,18 @@ kf_status launch_tc_linear(const void* X, long long ldx, const void* W, long lon
     if (grid_override > 0 && grid_override < grid) grid = grid_override - grid_override % cta_group;
     if (grid < cta_group) grid = cta_group;
     if (grid_out) *grid_out = grid;
-    const size_t fin_smem = (size_t)p.nsub * kFinWarps * sizeof(float2);
-    if (rn.norm != KF_NORM_NONE && fin_smem > 48 * 1024) return KF_ERR_UNSUPPORTED;   // N beyond 98304
+    // finishing pass: one warp per row keeps the most rows in flight (measured best on C4 and C5);
+    // more warps per row only for very long rows, whose coefficient table would not fit otherwise
+    int wpr = 1;
+    while (wpr < kFinWarps && (size_t)p.nsub * (kFinWarps / wpr) * sizeof(float2) > 40 * 1024) wpr <<= 1;
+    static const int env_wpr = [] {
+        const char* e = std::getenv("KF_FIN_WPR");
+        return e ? std::atoi(e) : 0;
+    }();
+    if (env_wpr == 1 || env_wpr == 2 || env_wpr == 4 || env_wpr == 8) wpr = env_wpr;
+    const int fin_rows = kFinWarps / wpr;
+    const size_t fin_smem = (size_t)p.nsub * fin_rows * sizeof(float2);
+    if (rn.norm != KF_NORM_NONE && fin_smem > 48 * 1024) return KF_ERR_UNSUPPORTED;   // N beyond ~780k
     if (cta_group == 2) {
         cudaLaunchConfig_t lc = {};
         lc.gridDim = dim3((unsigned)grid);
@@ -907,8 +941,8 @@ kf_status launch_tc_linear(const void* X, long long ldx, const void* W, long lon
     if (g_split_event && cudaEventRecord(g_split_event, st) != cudaSuccess) return KF_ERR_CUDA;
 
     if (rn.norm != KF_NORM_NONE) {
-        tc_rownorm_finish_kernel<<<(unsigned)((M + kFinWarps - 1) / kFinWarps), kFinWarps * 32, fin_smem, st>>>(
-            static_cast<__nv_bfloat16*>(Y), ldy, (int)M, (int)N, p.nsub, p.partials, rn.norm,
+        tc_rownorm_finish_kernel<<<(unsigned)((M + fin_rows - 1) / fin_rows), kFinWarps * 32, fin_smem, st>>>(
+            static_cast<__nv_bfloat16*>(Y), ldy, (int)M, (int)N, p.nsub, wpr, p.partials, rn.norm,
             static_cast<const __nv_bfloat16*>(rn.gamma), static_cast<const __nv_bfloat16*>(rn.beta), rn.eps);
         if (cudaGetLastError() != cudaSuccess) return KF_ERR_CUDA;
     }
