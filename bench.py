@@ -268,6 +268,19 @@ def run_kf(args):
                 torch.cuda.empty_cache()
         kf.check_device_status()
 
+    # ---------------------------------------------------------------- library GEMM under the same protocol
+    # (context only: an un-fused cuBLAS bf16 matmul of C3's shape, flushed and timed like the kf calls,
+    #  shows what the power-capped clocks of this run allow; it is not on any kf path)
+    live = None
+    if rank == 0 and not args.no_configs:
+        a = torch.randn(8192, 4096, device="cuda", dtype=torch.bfloat16)
+        b = torch.randn(4096, 4096, device="cuda", dtype=torch.bfloat16)
+        o = torch.empty(8192, 4096, device="cuda", dtype=torch.bfloat16)
+        lms, _ = time_steps(lambda: torch.matmul(a, b.t(), out=o), 20, 3, flush)
+        live = {"cublas_bf16_8192x4096x4096_ms": round(median(lms), 5),
+                "cublas_bf16_tflops": round(2 * 8192 * 4096 * 4096 / (median(lms) * 1e-3) / 1e12, 1)}
+        del a, b, o
+
     # ---------------------------------------------------------------- CPU baseline (oracle, rank 0, N == 1)
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
@@ -283,7 +296,7 @@ def run_kf(args):
                            "tile": {k: cfg[k] for k in ("kernel", "bm", "bn", "bk", "stages", "cta_group",
                                                         "epilogue_warps", "row_scheme", "grid")}},
                 "clocks": clk.summary(), "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
-                "cpu_baseline": cpu, "per_config": per_config,
+                "cpu_baseline": cpu, "per_config": per_config, "live_reference": live,
                 "frac_of_measured_burst": round(tflops / world / peaks["bf16_tflops"], 4),
                 "frac_of_nominal_2250": round(tflops / world / NOMINAL_TFLOPS, 4)}
         print(json.dumps(line))

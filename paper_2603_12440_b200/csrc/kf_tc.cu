@@ -10,7 +10,8 @@
 //               tcgen05.ld (one thread = one output row), bias (staged as fp32 in shared memory) /
 //               activation / scale / residual in fp32, per-row partial statistics of the 128-column
 //               sub-tile, 16-bit pack, 64-byte row segments stored straight from registers (shared
-//               memory is left to the operand ring: 7 stages of 32 KiB with CTA pairs)
+//               memory is left to the operand ring: 6 stages of 32 KiB with CTA pairs; a seventh
+//               stage measured no faster)
 // The two TMEM accumulators let the epilogue of tile i overlap the main loop of tile i+1.
 //
 // Row-norm (split-N): a row of N outputs spans N/128 sub-tiles owned by different warps and CTAs.  The epilogue
@@ -37,7 +38,7 @@ namespace kf {
 namespace {
 
 constexpr int BM = 128, BN = 256, BK = 64, UMMA_K = 16;
-constexpr int kMaxStages = 7;
+constexpr int kMaxStages = 6;
 constexpr int kEpiWarps = 8;                           // two per TMEM lane quarter, 128 columns each
 constexpr int kSub = BN / 2;                           // columns per epilogue warp = statistics sub-tile
 constexpr int kThreads = 32 * (2 + kEpiWarps);
@@ -47,15 +48,15 @@ constexpr uint32_t kABytes = BM * BK * 2;              // 16 KiB
 // CTAs of a cluster stage 128 rows of W each (16 KiB, 6 stages) and one tcgen05.mma.cta_group::2
 // of M = 256 reads both halves, which halves the shared-memory traffic per flop.
 template <int CG> struct Cfg {
-    static constexpr int kStages = CG == 2 ? 7 : 4;
+    static constexpr int kStages = CG == 2 ? 6 : 4;
     static constexpr uint32_t kBRows = BN / CG;
     static constexpr uint32_t kBBytes = kBRows * BK * 2;
     static constexpr uint32_t kStageBytes = kABytes + kBBytes;
     static constexpr uint32_t kSmemB = kStages * kABytes;
-    static_assert(kStages * kStageBytes <= 224 * 1024, "operand ring is at most 224 KiB");
+    static_assert(kStages * kStageBytes == 192 * 1024, "operand ring is 192 KiB in both modes");
 };
 constexpr uint32_t kSmemA = 0;
-constexpr uint32_t kSmemBias = 224 * 1024;             // 2 x BN floats (double buffered), behind the operand ring
+constexpr uint32_t kSmemBias = 192 * 1024;             // 2 x BN floats (double buffered), behind the operand ring
 constexpr uint32_t kSmemBar = kSmemBias + 2 * BN * 4;
 constexpr uint32_t kNumBars = 2 * kMaxStages + 6;         // ring full/empty, accumulator full/empty, bias ready
 constexpr uint32_t kSmemTmemPtr = kSmemBar + kNumBars * 8;
