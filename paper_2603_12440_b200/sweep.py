@@ -1,0 +1,66 @@
+"""Sweep the tunable choices of the tile table and print what each costs on a configuration.
+
+The paper's templated-kernel step (Section 3.4) instantiates a kernel for every parameter setting,
+times each and keeps the fastest; this is that step for the choices this library exposes:
+CTAs per MMA and grid size of the tensor-core kernel, and threads per row / ring on-off of the row
+kernels.  Each candidate runs in a fresh process (the overrides are read once per process):
+
+    python -m paper_2603_12440_b200.sweep --config c3 [--steps 30]
+
+Needs a B200; prints one JSON line per candidate and the winner.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent.parent
+
+
+def candidates(config: str):
+    if config == "c2":
+        yield {"KF_ROW_RING": "1"}, "ring kernel"
+        for tpr in (32, 64, 128, 256):
+            yield {"KF_ROW_RING": "0", "KF_ROW_TPR": str(tpr)}, f"register kernel, {tpr} threads per row"
+        return
+    if config == "c1":
+        yield {}, "table default"
+        yield {"KF_TILE_OVERRIDE": "kernel=2"}, "tiled CUDA-core kernel + row kernel"
+        return
+    for cg in (1, 2):
+        for grid in (0, 144, 128, 112, 96):
+            ov = f"cg={cg}" + (f",grid={grid}" if grid else "")
+            yield {"KF_TILE_OVERRIDE": ov}, ov
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--config", default="c3", choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--steps", type=int, default=30)
+    args = ap.parse_args()
+    results = []
+    for env_add, label in candidates(args.config):
+        env = dict(os.environ)
+        env.update(env_add)
+        out = subprocess.run([sys.executable, str(ROOT / "bench.py"), "--only", args.config, "--steps",
+                              str(args.steps), "--warmup", "3"], env=env, capture_output=True, text=True)
+        line = out.stdout.strip().splitlines()[-1] if out.returncode == 0 and out.stdout.strip() else None
+        rec = {"candidate": label, "env": env_add}
+        if line:
+            rec.update(json.loads(line))
+        else:
+            rec["error"] = (out.stderr or "").strip().splitlines()[-1:] or ["failed"]
+        results.append(rec)
+        print(json.dumps(rec), flush=True)
+    ok = [r for r in results if "ms_median" in r]
+    if ok:
+        best = min(ok, key=lambda r: r["ms_median"])
+        print(json.dumps({"winner": best["candidate"], "ms_median": best["ms_median"], "config": args.config}))
+
+
+if __name__ == "__main__":
+    main()
