@@ -305,7 +305,7 @@ def run_kf(args):
 
 
 # DRAM bytes per launch from ncu captures (dram__bytes_read.sum + dram__bytes_write.sum); see profiles/
-TRAFFIC = {"c4_main": None}
+TRAFFIC = {"c4_main": 87432960}      # 52.82 MB read + 34.61 MB written (part of Y still dirty in L2 at kernel end)
 
 
 # ------------------------------------------------------------------------------------------ CPU arms

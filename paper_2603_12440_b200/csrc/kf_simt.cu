@@ -54,17 +54,16 @@ simt_rows_kernel(const T* __restrict__ X, long long ldx, const T* __restrict__ W
         for (int j = 0; j < NPT; ++j) {
             if (j > 0) __syncthreads();
             // slab j: W rows j*256 .. j*256+255, k0 .. k0+31; a warp reads one row per step (coalesced)
-            // 32 rows per warp; the loads are independent, so issue them in batches of 8 before storing
+            // 32 rows per warp; the loads are independent, so all are issued before the first store
+            {
+                float tmp[32];
 #pragma unroll
-            for (int r0 = 0; r0 < kThreads; r0 += 8 * (kThreads / 32)) {
-                float tmp[8];
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const int n = j * kThreads + r0 + u * (kThreads / 32) + warp;
+                for (int u = 0; u < 32; ++u) {
+                    const int n = j * kThreads + u * (kThreads / 32) + warp;
                     tmp[u] = (n < N && k0 + lane < K) ? Elem<T>::load(W + (long long)n * ldw + k0 + lane) : 0.f;
                 }
 #pragma unroll
-                for (int u = 0; u < 8; ++u) ws[r0 + u * (kThreads / 32) + warp][lane] = tmp[u];
+                for (int u = 0; u < 32; ++u) ws[u * (kThreads / 32) + warp][lane] = tmp[u];
             }
             __syncthreads();
 #pragma unroll

@@ -60,8 +60,8 @@ constexpr uint32_t kSmemBias = 192 * 1024;             // 2 x BN floats (double 
 constexpr uint32_t kSmemBar = kSmemBias + 2 * BN * 4;
 constexpr uint32_t kNumBars = 2 * kMaxStages + 6;         // ring full/empty, accumulator full/empty, bias ready
 constexpr uint32_t kSmemTmemPtr = kSmemBar + kNumBars * 8;
-constexpr uint32_t kSmemAbort = kSmemTmemPtr + 4;
-constexpr uint32_t kSmemAlloc = kSmemAbort + 4;
+constexpr uint32_t kSmemAbort = kSmemTmemPtr + 8;      // abort flag (4 B, 8-byte aligned), then the wait limit (8 B)
+constexpr uint32_t kSmemAlloc = kSmemAbort + 16;
 static_assert(kSmemAlloc <= 232448, "exceeds the 227 KiB per-CTA shared memory of sm_100");
 
 constexpr long long kTimeoutCycles = 3000000000ll;     // about 1.5-2 s: far above any legitimate wait
@@ -93,12 +93,13 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 // bounded wait: false = gave up (status recorded, abort raised) or another role aborted
 __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
                                             uint32_t* status, uint32_t code) {
+    const long long limit = *reinterpret_cast<volatile long long*>(const_cast<uint32_t*>(abort_flag) + 2);
     const long long t0 = clock64();
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 0x3F) == 0) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > kTimeoutCycles) {
+            if (clock64() - t0 > limit) {
                 *abort_flag = 1;
                 if (atomicCAS(status, 0u, (uint32_t)KF_ERR_TIMEOUT) == 0u) status[1] = code;
                 __threadfence();
@@ -272,7 +273,9 @@ struct TcParams {
     uint32_t* status;
     __nv_bfloat16* Y;           // output (or 16-bit intermediate), row pitch ldy
     long long ldy;
-    int debug;                  // timing experiments only (results are wrong): 1 no TMA loads, 2 no MMAs, 4 no epilogue work
+    int debug;                  // timing experiments only (results are wrong): 1 no TMA loads, 2 no MMAs, 4 no epilogue work;
+                                // 512 = the producer never signals, so every wait runs into its limit (time-out test)
+    long long timeout_cycles;   // limit of every bounded wait
 };
 
 // element-wise epilogue on 32 consecutive columns of one row, fast-math forms (bf16 output).
@@ -387,6 +390,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             mbar_init(bias_bar(a), kEpiWarps);
         }
         *abort_flag = 0;
+        *reinterpret_cast<volatile long long*>(smem_raw + kSmemAbort + 8) = p.timeout_cycles;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -414,6 +418,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             uint32_t stage = 0, phase = 0;
             bool ok = true;
             for (int tile = unit; tile < num_tiles && ok; tile += num_units) {
+                if (p.debug & 512) break;                  // time-out test: nothing is ever loaded or signalled
                 const int mb = (tile / p.tiles_n) * CG + (int)rank, nb = tile % p.tiles_n;
                 for (int kb = 0; kb < kblocks; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 0x100u + stage)) { ok = false; break; }
@@ -901,6 +906,12 @@ kf_status launch_tc_linear(const void* X, long long ldx, const void* W, long lon
         return e ? std::atoi(e) : 0;
     }();
     p.debug = debug_mode;
+    static const long long timeout_cycles = [] {           // KF_TC_TIMEOUT_MS shortens the limit (tests)
+        const char* e = std::getenv("KF_TC_TIMEOUT_MS");
+        const long long ms = e ? std::atoll(e) : 0;
+        return ms > 0 ? ms * 2000000ll : kTimeoutCycles;    // ~2 GHz clock64
+    }();
+    p.timeout_cycles = timeout_cycles;
 
     int grid = tc_default_grid(M, N, cta_group);
     if (grid_override > 0 && grid_override < grid) grid = grid_override - grid_override % cta_group;

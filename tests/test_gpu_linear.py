@@ -226,3 +226,35 @@ def test_degenerate_sizes(kf):
     assert np.all(run(kf, one) == 1.0)
     ln1 = make("f32", 40, 1, 16, seed=35, norm="layernorm")
     assert_parity(run(kf, ln1), oracle_of(ln1), "f32", "N=1 layernorm = beta")
+
+
+def test_tc_random_shapes_and_options(kf):
+    """Seeded random draw of shapes (ragged in every dimension, multiples of 8 as the tensor-core path
+    needs) and of every epilogue / row-op option, each compared with the oracle."""
+    r = np.random.Generator(np.random.PCG64(77))
+    for i in range(14):
+        M = int(r.integers(1, 700))
+        N = 8 * int(r.integers(1, 300))
+        K = 8 * int(r.integers(1, 70))
+        act = ACTS[int(r.integers(0, len(ACTS)))]
+        norm = ["none", "softmax", "layernorm", "rmsnorm"][int(r.integers(0, 4))]
+        p = make("bf16", M, N, K, seed=1000 + i, act=act, norm=norm, bias=bool(r.integers(0, 2)),
+                 res=bool(r.integers(0, 2)), scale=float(r.choice([1.0, 0.5, 2.0])))
+        assert kf.tile_config(M, N, K, torch.bfloat16, norm)["kernel"] == 3
+        assert_parity(run(kf, p), oracle_of(p), "bf16", f"random {i}: {M}x{N}x{K} {act} {norm}")
+
+
+def test_concat_x_layernorm_x_layout(kf):
+    """out = concat(x, layer_norm(x)) along the columns: the row op writes straight into the right half of
+    the wider buffer through its row pitch (one of the paper's custom operators, Section 4.4)."""
+    r = np.random.Generator(np.random.PCG64(78))
+    M, N = 900, 1024
+    X = inputs._store(r.standard_normal((M, N)) * 2 + 1, "bf16")
+    g = inputs._store(1 + 0.1 * r.standard_normal(N), "bf16")
+    b = inputs._store(0.1 * r.standard_normal(N), "bf16")
+    dX, dg, db = to_device(X, "bf16"), to_device(g, "bf16"), to_device(b, "bf16")
+    out = torch.zeros(M, 2 * N, dtype=torch.bfloat16, device="cuda")
+    out[:, :N] = dX
+    kf.row_layernorm(dX, dg, db, 1e-5, out=out[:, N:])
+    assert torch.equal(out[:, :N], dX)
+    assert_parity(to_f64(out[:, N:]), kfo.row_layernorm(X, g, b, 1e-5), "bf16", "concat layout")

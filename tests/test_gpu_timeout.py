@@ -1,0 +1,43 @@
+"""Failure detection on the device without a fault: every wait inside the tensor-core kernel is
+bounded.  A test switch makes the producer warp never signal, so each wait runs into its (shortened)
+limit; the kernel must record KF_ERR_TIMEOUT in the workspace status word, return, and leave the
+context usable.  Runs in a child process because the switches are read once per process."""
+import os
+import subprocess
+import sys
+from pathlib import Path
+
+import pytest
+
+ROOT = Path(__file__).resolve().parent.parent
+
+CHILD = r"""
+import sys
+sys.path.insert(0, %r)
+import torch
+import paper_2603_12440_b200 as kf
+x = torch.randn(300, 256, device="cuda", dtype=torch.bfloat16)
+w = torch.randn(520, 256, device="cuda", dtype=torch.bfloat16)
+y = kf.linear_epilogue_rownorm(x, w, norm="softmax")
+try:
+    kf.check_device_status()
+    print("NO_ERROR")
+except kf.KfError as e:
+    print("STATUS", e.status)
+# the status word was cleared by the check, and the context still works
+kf.check_device_status()
+z = kf.row_softmax(torch.randn(64, 512, device="cuda"))
+torch.cuda.synchronize()
+print("ROWSUM", float(z.sum(1).mean()))
+"""
+
+
+@pytest.mark.gpu
+def test_bounded_waits_report_a_timeout_and_the_context_survives():
+    env = dict(os.environ, KF_TC_DEBUG="512", KF_TC_TIMEOUT_MS="150")
+    out = subprocess.run([sys.executable, "-c", CHILD % str(ROOT)], env=env, capture_output=True, text=True, timeout=240)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = out.stdout.strip().splitlines()
+    assert "STATUS 6" in lines, out.stdout          # KF_ERR_TIMEOUT
+    rowsum = [l for l in lines if l.startswith("ROWSUM")]
+    assert rowsum and abs(float(rowsum[0].split()[1]) - 1.0) < 1e-5
