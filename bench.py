@@ -280,6 +280,14 @@ def run_kf(args):
         live = {"cublas_bf16_8192x4096x4096_ms": round(median(lms), 5),
                 "cublas_bf16_tflops": round(2 * 8192 * 4096 * 4096 / (median(lms) * 1e-3) / 1e12, 1)}
         del a, b, o
+        # a plain device copy of C2's size (128 MiB in, 128 MiB out), timed the same way: what HBM gives a
+        # transfer this short (the 6.5 TB/s copy peak is only reached on multi-GiB copies)
+        cx = torch.empty(16384, 4096, device="cuda", dtype=torch.bfloat16).normal_()
+        cy = torch.empty_like(cx)
+        cms, _ = time_steps(lambda: cy.copy_(cx), 20, 3, flush)
+        live["copy_128MiB_ms"] = round(median(cms), 5)
+        live["copy_128MiB_GBs"] = round(2 * cx.numel() * 2 / (median(cms) * 1e-3) / 1e9, 1)
+        del cx, cy
 
     # ---------------------------------------------------------------- CPU baseline (oracle, rank 0, N == 1)
     cpu = None

@@ -207,23 +207,7 @@ row_norm_ring_kernel(const T* X, long long ldx, T* Y, long long ldy, long long M
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    // gamma / beta as fp32, de-interleaved so that a lane's two float4 halves are conflict-free reads
-    if (NORM != KF_NORM_SOFTMAX) {
-        for (int idx = threadIdx.x; idx < NV; idx += kRingThreads) {
-            float g[E], b[E];
-#pragma unroll
-            for (int e = 0; e < E; ++e) { g[e] = 1.f; b[e] = 0.f; }
-            if (gamma) unpack<T>(__ldg(reinterpret_cast<const uint4*>(gamma) + idx), g);
-            if (beta && NORM == KF_NORM_LAYERNORM) unpack<T>(__ldg(reinterpret_cast<const uint4*>(beta) + idx), b);
-#pragma unroll
-            for (int h = 0; h < E / 4; ++h) {
-                gam[h * NV + idx] = make_float4(g[h * 4], g[h * 4 + 1], g[h * 4 + 2], g[h * 4 + 3]);
-                if (NORM == KF_NORM_LAYERNORM)
-                    bet[h * NV + idx] = make_float4(b[h * 4], b[h * 4 + 1], b[h * 4 + 2], b[h * 4 + 3]);
-            }
-        }
-    }
-    __syncthreads();
+    __syncthreads();                                     // barriers exist; the producer starts at once
 
     // rows of this CTA: blockIdx.x, blockIdx.x + gridDim.x, ...; its i-th row uses slot i % slots
     const long long my_rows = (M - blockIdx.x + gridDim.x - 1) / gridDim.x;
@@ -240,6 +224,25 @@ row_norm_ring_kernel(const T* X, long long ldx, T* Y, long long ldy, long long M
             }
         }
         return;
+    }
+
+    // consumers, while the first rows are in flight: gamma / beta as fp32, de-interleaved so that a
+    // lane's two float4 halves are conflict-free reads; then a barrier among the consumer warps only
+    if (NORM != KF_NORM_SOFTMAX) {
+        for (int idx = threadIdx.x; idx < NV; idx += kRingConsumers * 32) {
+            float g[E], b[E];
+#pragma unroll
+            for (int e = 0; e < E; ++e) { g[e] = 1.f; b[e] = 0.f; }
+            if (gamma) unpack<T>(__ldg(reinterpret_cast<const uint4*>(gamma) + idx), g);
+            if (beta && NORM == KF_NORM_LAYERNORM) unpack<T>(__ldg(reinterpret_cast<const uint4*>(beta) + idx), b);
+#pragma unroll
+            for (int h = 0; h < E / 4; ++h) {
+                gam[h * NV + idx] = make_float4(g[h * 4], g[h * 4 + 1], g[h * 4 + 2], g[h * 4 + 3]);
+                if (NORM == KF_NORM_LAYERNORM)
+                    bet[h * NV + idx] = make_float4(b[h * 4], b[h * 4 + 1], b[h * 4 + 2], b[h * 4 + 3]);
+            }
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(kRingConsumers * 32) : "memory");
     }
 
     for (long long i = warp; i < my_rows; i += kRingConsumers) {
