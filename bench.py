@@ -148,6 +148,18 @@ def median(v):
     return s[len(s) // 2]
 
 
+def aggregate_replicas(ms_local: float, flops_per_rank: int, world: int, device="cuda"):
+    """Whole-job rate of `world` independent replicas: (max step time over ranks, total TFLOP/s).
+    The only collective of the multi-GPU path; works on any backend (NCCL on GPUs, gloo in the CPU test)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_max = float(t.item())
+    return ms_max, world * flops_per_rank / (ms_max * 1e-3) / 1e12
+
+
 def run_kf(args):
     import torch
     import torch.distributed as dist
@@ -200,11 +212,7 @@ def run_kf(args):
         barrier()
     kf.check_device_status()
     ms = sum(total_ms) / len(total_ms)
-    t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_max = float(t.item())
-    tflops = world * p.flops / (ms_max * 1e-3) / 1e12
+    ms_max, tflops = aggregate_replicas(ms, p.flops, world)
 
     main_avg = sum(main_ms) / len(main_ms)
     achieved = p.flops / (main_avg * 1e-3) / 1e12
@@ -231,13 +239,11 @@ def run_kf(args):
         barrier()
         e_ms, _ = time_steps(host_call, e_steps, 3, flush)
         barrier()
-        te = torch.tensor([sum(e_ms) / len(e_ms)], dtype=torch.float64, device="cuda")
-        if world > 1:
-            dist.all_reduce(te, op=dist.ReduceOp.MAX)
+        e_max, e_tflops = aggregate_replicas(sum(e_ms) / len(e_ms), p.flops, world)
         h2d = sum(v.numel() * v.element_size() for v in (h["X"], h["W"], h["bias"], h["gamma"], h["beta"]))
-        e2e = {"value": round(world * p.flops / (float(te.item()) * 1e-3) / 1e12, 3), "unit": "TFLOP/s",
+        e2e = {"value": round(e_tflops, 3), "unit": "TFLOP/s",
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(hout.numel() * 2),
-               "ms_per_step": round(float(te.item()), 4), "steps": e_steps,
+               "ms_per_step": round(e_max, 4), "steps": e_steps,
                "api": "kf_linear_epilogue_rownorm_host (pinned host buffers in, pinned host Y out)"}
         del arena, h, hout
 
