@@ -29,6 +29,10 @@
  *     kf_check_device_status.  Calls that share a `ws` must not overlap on the GPU.
  *   - Alignment: fast paths need 16-byte aligned base pointers and row pitches; anything else
  *     is served by slower generic kernels, never by the CPU.  There is no CPU fallback.
+ *   - fp32 calls never take a single TF32 pass (10 mantissa bits miss the 1e-4 gate): small or
+ *     unaligned ones run on CUDA cores, large aligned ones (M > 128, 2MNK >= 4e9) on the tensor
+ *     cores through three error-compensated TF32 passes with K accumulated in fp32-summed chunks;
+ *     those need ws room for hi / lo copies of X and W (kf_workspace_bytes accounts for it).
  *   - M == 0 or N == 0: returns KF_OK and writes nothing.  K == 0: the accumulator is 0.
  *   - Aliasing: Y may alias residual (same pitch) and, for the row functions, X.  Y must not
  *     overlap X or W of the linear calls.  Inputs must be finite.
@@ -93,7 +97,7 @@ typedef struct {
 /* Which kernel and tile shape a call resolves to (the hardware-aware table, Section 3.4:
  * the best-measured instantiation of a templated kernel is the one that is used). */
 typedef struct {
-    int32_t kernel;           /* 0 none, 1 SIMT row-resident, 2 SIMT tiled, 3 tcgen05 */
+    int32_t kernel;           /* 0 none, 1 SIMT row-resident, 2 SIMT tiled, 3 tcgen05 bf16, 4 tcgen05 fp32 (3xTF32) */
     int32_t bm, bn, bk;       /* tile of one work unit (a CTA, or a CTA pair when cta_group is 2) */
     int32_t stages;           /* shared-memory pipeline depth */
     int32_t cta_group;        /* 1 or 2 CTAs per MMA */
@@ -165,8 +169,10 @@ size_t kf_host_call_bytes(int64_t M, int64_t N, int64_t K, kf_dtype dt, int has_
  * Same arguments, results and kernels as kf_linear_epilogue_rownorm, minus ws / ws_bytes.
  *   - Limit: kf_workspace_bytes(M,N,K,dt,norm) must not exceed 8 MiB + 256 bytes, i.e. a bf16
  *     row-norm may span at most 2048 output tiles of 128 x 256 (ceil(M/128) * ceil(N/256)).  Larger
- *     problems return KF_ERR_SCRATCH_LIMIT and launch nothing.  Calls without a row-norm and fp32
- *     calls need only the status block and are never rejected for size.
+ *     problems return KF_ERR_SCRATCH_LIMIT and launch nothing.  bf16 calls without a row-norm and
+ *     small fp32 calls need only the status block; a large aligned fp32 call, which the normal form
+ *     would run on the tensor cores, needs room for the split operands (kf_workspace_bytes says how
+ *     much) and is rejected here once that exceeds the limit.
  *   - Every device that loads the library holds the 8 MiB array until the process exits.
  *   - The call performs no cudaMalloc / cudaFree and calls no allocating routine.  The first call
  *     on each device looks the array's device address up (cudaGetSymbolAddress, with that device

@@ -13,8 +13,8 @@ from pathlib import Path
 PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libkf.so"
-SOURCES = ["kf_api.cu", "kf_row.cu", "kf_simt.cu", "kf_tc.cu"]
-HEADERS = ["kf_common.cuh", "kf_tc.cuh", "../../include/kf.h"]
+SOURCES = ["kf_api.cu", "kf_row.cu", "kf_simt.cu", "kf_tc.cu", "kf_tc32.cu"]
+HEADERS = ["kf_common.cuh", "kf_tc.cuh", "kf_tc_ptx.cuh", "../../include/kf.h"]
 
 
 def nvcc_path() -> str:

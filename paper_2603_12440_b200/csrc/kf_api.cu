@@ -53,6 +53,14 @@ kf_status resolve(long long M, long long N, long long K, int dt, int norm, bool 
         if (c->grid < c->cta_group) c->grid = c->cta_group;
         return KF_OK;
     }
+    // large aligned fp32: tensor cores through three TF32 passes; the row op then runs in place on the fp32 result
+    if (dt == KF_F32 && aligned && tc32_shape_ok(M, N, K) && ov.kernel != 1 && ov.kernel != 2) {
+        c->kernel = 4;
+        c->bm = 256; c->bn = 256; c->bk = 32; c->stages = 3; c->cta_group = 2; c->epilogue_warps = 8;
+        c->row_scheme = norm == KF_NORM_NONE ? 0 : 4;
+        c->grid = tc32_default_grid(M, N);
+        return KF_OK;
+    }
     bool rows = simt_row_resident_ok(N) && (norm != KF_NORM_NONE ? (M < 4096 || dt == KF_BF16) : (M <= 1024));
     if (ov.kernel == 1 && simt_row_resident_ok(N)) rows = true;
     if (ov.kernel == 2 && (norm == KF_NORM_NONE || dt == KF_F32)) rows = false;
@@ -121,6 +129,18 @@ kf_status linear_impl(const void* X, int64_t ldx, const void* W, int64_t ldw, vo
         if (!ws || ws_bytes < need) return KF_ERR_WORKSPACE;
         return launch_tc_linear(X, ldx, W, ldw, Y, ldy, M, N, K, ep, rn, ws, cfg.cta_group, env_override().grid, st, nullptr);
     }
+    // the 3xTF32 kernel keeps running sums of K chunks in Y, so a residual that aliases Y goes to CUDA cores
+    if (cfg.kernel == 4 && ep.residual == Y) {
+        cfg.kernel = 2;
+        cfg.row_scheme = rn.norm == KF_NORM_NONE ? 0 : 4;
+    }
+    if (cfg.kernel == 4) {
+        const size_t need = kStatusBytes + tc32_split_bytes(M, N, K);
+        if (!ws || ws_bytes < need) return KF_ERR_WORKSPACE;
+        s = launch_tc32_linear(X, ldx, W, ldw, Y, ldy, M, N, K, ep, ws, st, nullptr);
+        if (s != KF_OK || rn.norm == KF_NORM_NONE) return s;
+        return launch_row_norm(Y, ldy, Y, ldy, M, N, dt, rn, st) == cudaSuccess ? KF_OK : KF_ERR_CUDA;
+    }
     cudaError_t e = launch_simt_linear(X, ldx, W, ldw, Y, ldy, M, N, K, dt, ep, rn, cfg.kernel == 1, st, nullptr);
     return e == cudaSuccess ? KF_OK : KF_ERR_CUDA;
 }
@@ -178,6 +198,7 @@ size_t kf_workspace_bytes(int64_t M, int64_t N, int64_t K, kf_dtype dt, kf_norm 
     (void)K;
     size_t b = kStatusBytes;
     if (dt == KF_BF16 && norm != KF_NORM_NONE && M > 0 && N > 0) b += tc_partials_bytes(M, N);
+    if (dt == KF_F32 && M > 0 && N > 0 && tc32_shape_ok(M, N, K)) b += tc32_split_bytes(M, N, K);
     return round256(b);
 }
 

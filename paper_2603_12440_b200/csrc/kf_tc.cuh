@@ -22,6 +22,16 @@ kf_status launch_tc_linear(const void* X, long long ldx, const void* W, long lon
 kf_status tc_static_scratch(void** ptr);
 size_t tc_static_scratch_bytes();
 
+// fp32 through three TF32 tensor-core passes (kf_tc32.cu): shapes served, workspace behind the status
+// block for the hi / lo operand copies, grid, launcher (element-wise epilogue only; X, W, Y, residual
+// 16-byte aligned, K and N multiples of 4)
+bool tc32_shape_ok(long long M, long long N, long long K);
+size_t tc32_split_bytes(long long M, long long N, long long K);
+int tc32_default_grid(long long M, long long N);
+kf_status launch_tc32_linear(const void* X, long long ldx, const void* W, long long ldw, void* Y, long long ldy,
+                             long long M, long long N, long long K, const EpilogueParams& ep, void* ws,
+                             cudaStream_t st, int* grid_out);
+
 // profiling aid: event recorded between the GEMM kernel and the finishing kernel (nullptr = off)
 void tc_set_split_event(cudaEvent_t ev);
 

@@ -70,8 +70,14 @@ def test_tile_table_on_the_five_configs(kf):
     with pytest.raises(kf.KfError) as e:
         kf.tile_config(512, 4104, 520, torch.bfloat16, "softmax", aligned=False)
     assert e.value.status == 2
-    # fp32 never goes to the tensor cores
-    assert kf.tile_config(8192, 8192, 8192, torch.float32, "none")["kernel"] == 2
+    # fp32 never takes a single TF32 pass: small or unaligned shapes stay on CUDA cores, large aligned ones
+    # go through three error-compensated TF32 passes (kernel 4), the row op then runs in place (scheme 4)
+    big = kf.tile_config(8192, 8192, 8192, torch.float32, "softmax")
+    assert (big["kernel"], big["bm"], big["bn"], big["bk"], big["stages"], big["cta_group"], big["row_scheme"]) == \
+        (4, 256, 256, 32, 3, 2, 4)
+    assert kf.tile_config(8192, 8192, 8192, torch.float32, "none", aligned=False)["kernel"] == 2
+    assert kf.tile_config(8192, 8192, 8190, torch.float32, "none")["kernel"] == 2
+    assert kf.workspace_bytes(8192, 8192, 8192, torch.float32, "none") == 256 + 4 * 8192 * 8192 * 4
     assert kf.tile_config(0, 8192, 8192, torch.float32, "none")["kernel"] == 0
 
 

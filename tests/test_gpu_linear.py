@@ -258,3 +258,28 @@ def test_concat_x_layernorm_x_layout(kf):
     kf.row_layernorm(dX, dg, db, 1e-5, out=out[:, N:])
     assert torch.equal(out[:, :N], dX)
     assert_parity(to_f64(out[:, N:]), kfo.row_layernorm(X, g, b, 1e-5), "bf16", "concat layout")
+
+
+# ------------------------------------------------------------------------------- fp32 (tcgen05, 3xTF32)
+def test_tc32_small_integers_are_exact(kf):
+    """fp32 on the tensor cores through three TF32 passes: integer operands are exact in TF32, so the
+    result must equal the oracle bit for bit (2 x 5 tiles, ragged in M, N and K)."""
+    r = np.random.Generator(np.random.PCG64(91))
+    M, N, K = 200, 1028, 10004
+    X = r.integers(-3, 4, (M, K)).astype(np.float32)
+    W = r.integers(-3, 4, (N, K)).astype(np.float32)
+    assert kf.tile_config(M, N, K, torch.float32, "none")["kernel"] == 4
+    y = kf.linear_epilogue(to_device(X, "f32"), to_device(W, "f32"))
+    kf.check_device_status()
+    assert np.array_equal(to_f64(y), kfo.linear_epilogue(X, W))
+
+
+@pytest.mark.parametrize("norm", ["none", "softmax", "layernorm"])
+def test_tc32_matches_oracle_under_the_fp32_gate(kf, norm):
+    # full-mantissa fp32 operands: a single TF32 pass would miss the 1e-4 gate by an order of magnitude
+    M, N, K = 515, 1028, 4100
+    p = make("f32", M, N, K, seed=92, act="gelu_erf", norm=norm, res=True, scale=0.5)
+    cfg = kf.tile_config(M, N, K, torch.float32, norm)
+    assert cfg["kernel"] == 4 and cfg["row_scheme"] == (0 if norm == "none" else 4)
+    r = assert_parity(run(kf, p), oracle_of(p), "f32", f"tc32 {norm}")
+    assert r["max_abs"] < 2e-5

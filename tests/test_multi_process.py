@@ -24,10 +24,17 @@ dist.destroy_process_group()
 """
 
 
+def _free_port():
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
 def _torchrun(args, env_extra=None):
     env = dict(os.environ, **(env_extra or {}))
     cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2",
-           "--master-addr", "127.0.0.1", "--master-port", "29731"] + args
+           "--master-addr", "127.0.0.1", "--master-port", str(_free_port())] + args
     return subprocess.run(cmd, capture_output=True, text=True, timeout=600, env=env, cwd=str(ROOT))
 
 
