@@ -19,7 +19,8 @@ rank, world = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"])
 dist.init_process_group("gloo")
 ms_local = 0.2 if rank == 0 else 0.5          # the slower rank sets the job's step time
 ms_max, tflops = bench.aggregate_replicas(ms_local, 10**12, world, device="cpu")
-print(json.dumps({"rank": rank, "ms_max": ms_max, "tflops": tflops}))
+with open(os.path.join(%r, "rank%%d.json" %% rank), "w") as f:     # one file per rank: stdout of ranks can interleave
+    json.dump({"rank": rank, "ms_max": ms_max, "tflops": tflops}, f)
 dist.destroy_process_group()
 """
 
@@ -40,10 +41,10 @@ def _torchrun(args, env_extra=None):
 
 def test_replica_aggregation_takes_the_max_over_ranks(tmp_path):
     script = tmp_path / "worker.py"
-    script.write_text(WORKER % str(ROOT))
+    script.write_text(WORKER % (str(ROOT), str(tmp_path)))
     out = _torchrun([str(script)])
     assert out.returncode == 0, out.stderr[-2000:]
-    recs = [json.loads(l) for l in out.stdout.splitlines() if l.startswith("{")]
+    recs = [json.loads((tmp_path / f"rank{r}.json").read_text()) for r in (0, 1)]
     assert sorted(r["rank"] for r in recs) == [0, 1]
     for r in recs:
         assert r["ms_max"] == 0.5
