@@ -274,6 +274,46 @@ def run_kf(args):
                 torch.cuda.empty_cache()
         kf.check_device_status()
 
+    # ---------------------------------------------------------------- further kf calls (not gating)
+    # stand-alone row softmax at two shapes, the un-fused forms of C4 / C5 (linear + epilogue, then the row
+    # kernel in place: what fusing the row statistics saves), and a large fp32 call (3xTF32 tensor-core path)
+    extras = {}
+    if rank == 0 and not args.no_configs:
+        def timed(fn, steps=15):
+            tms, _ = time_steps(fn, steps, 3, flush)
+            return round(median(tms), 5)
+        for (m_, n_) in ((2048, 32768), (16384, 4096)):
+            xs = torch.randn(m_, n_, device="cuda", dtype=torch.bfloat16)
+            ys = torch.empty_like(xs)
+            ms_ = timed(lambda: kf.row_softmax(xs, out=ys))
+            extras[f"row_softmax_bf16_{m_}x{n_}"] = {"ms_median": ms_, "GB/s": round(2 * xs.numel() * 2 / (ms_ * 1e-3) / 1e9, 1)}
+            del xs, ys
+        for idx in (4, 5):
+            q = p if idx == 4 else inputs.config(5)
+            dq = d if idx == 4 else device_problem(q)
+            yq = torch.empty((q.M, q.N), dtype=torch.bfloat16, device="cuda")
+
+            def unfused():
+                kf.linear_epilogue(dq["X"], dq["W"], dq["bias"], q.act, q.scale, dq["residual"], out=yq)
+                if q.norm == "softmax":
+                    kf.row_softmax(yq, out=yq)
+                else:
+                    kf.row_layernorm(yq, dq["gamma"], dq["beta"], q.eps, out=yq)
+            extras[f"C{idx}_unfused_linear_then_row_kernel"] = {
+                "ms_median": timed(unfused), "note": "pre-norm row rounded to bf16 between the two kernels"}
+            del yq
+            if idx != 4:
+                del dq
+        xf = torch.randn(4096, 4096, device="cuda")
+        wf = torch.randn(4096, 4096, device="cuda") / 64
+        yf = torch.empty(4096, 4096, device="cuda")
+        ms_ = timed(lambda: kf.linear_epilogue(xf, wf, out=yf), 8)
+        extras["f32_linear_4096x4096x4096_3xTF32"] = {"ms_median": ms_, "TFLOP/s": round(2 * 4096 ** 3 / (ms_ * 1e-3) / 1e12, 1),
+                                                      "tile": kf.tile_config(4096, 4096, 4096, torch.float32, "none")}
+        del xf, wf, yf
+        torch.cuda.empty_cache()
+        kf.check_device_status()
+
     # ---------------------------------------------------------------- library GEMM under the same protocol
     # (context only: an un-fused cuBLAS bf16 matmul of C3's shape, flushed and timed like the kf calls,
     #  shows what the power-capped clocks of this run allow; it is not on any kf path)
@@ -310,7 +350,7 @@ def run_kf(args):
                            "tile": {k: cfg[k] for k in ("kernel", "bm", "bn", "bk", "stages", "cta_group",
                                                         "epilogue_warps", "row_scheme", "grid")}},
                 "clocks": clk.summary(), "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
-                "cpu_baseline": cpu, "per_config": per_config, "live_reference": live,
+                "cpu_baseline": cpu, "per_config": per_config, "extras": extras, "live_reference": live,
                 "frac_of_measured_burst": round(tflops / world / peaks["bf16_tflops"], 4),
                 "frac_of_nominal_2250": round(tflops / world / NOMINAL_TFLOPS, 4)}
         print(json.dumps(line))

@@ -71,7 +71,7 @@ row_norm_reg_kernel(const T* X, long long ldx, T* Y, long long ldy, long long M,
             if (lr + i * tpr < NV) {
                 unpack<T>(v[i], f);
 #pragma unroll
-                for (int e = 0; e < E; ++e) s += exp2f(fmaf(f[e], kLog2e, -ms));
+                for (int e = 0; e < E; ++e) s += fast_ex2(fmaf(f[e], kLog2e, -ms));
             }
         s = group_reduce<false>(s, tpr, red);
         const float inv = 1.0f / s;
@@ -81,7 +81,7 @@ row_norm_reg_kernel(const T* X, long long ldx, T* Y, long long ldy, long long M,
             if (live && idx < NV) {
                 unpack<T>(v[i], f);
 #pragma unroll
-                for (int e = 0; e < E; ++e) f[e] = exp2f(fmaf(f[e], kLog2e, -ms)) * inv;
+                for (int e = 0; e < E; ++e) f[e] = fast_ex2(fmaf(f[e], kLog2e, -ms)) * inv;
                 st_stream(yr + idx, pack<T>(f));
             }
         }
@@ -271,7 +271,7 @@ row_norm_ring_kernel(const T* X, long long ldx, T* Y, long long ldy, long long M
                 if (lane + v * 32 < NV) {
                     unpack<T>(srow[lane + v * 32], x);
 #pragma unroll
-                    for (int e = 0; e < E; ++e) l[e & 3] += exp2f(fmaf(x[e], kLog2e, -ms));
+                    for (int e = 0; e < E; ++e) l[e & 3] += fast_ex2(fmaf(x[e], kLog2e, -ms));
                 }
             const float inv = 1.0f / warp_sum((l[0] + l[1]) + (l[2] + l[3]));
 #pragma unroll
@@ -280,7 +280,7 @@ row_norm_ring_kernel(const T* X, long long ldx, T* Y, long long ldy, long long M
                 if (idx < NV) {
                     unpack<T>(srow[idx], x);
 #pragma unroll
-                    for (int e = 0; e < E; ++e) x[e] = exp2f(fmaf(x[e], kLog2e, -ms)) * inv;
+                    for (int e = 0; e < E; ++e) x[e] = fast_ex2(fmaf(x[e], kLog2e, -ms)) * inv;
                     st_stream(yr + idx, pack<T>(x));
                 }
             }
@@ -346,11 +346,11 @@ row_norm_generic_kernel(const T* X, long long ldx, T* Y, long long ldy, long lon
         for (long long n = threadIdx.x; n < N; n += tpr) m = fmaxf(m, Elem<T>::load(xr + n));
         m = group_reduce<true>(m, tpr, red);
         float s = 0.f;
-        for (long long n = threadIdx.x; n < N; n += tpr) s += exp2f((Elem<T>::load(xr + n) - m) * kLog2e);
+        for (long long n = threadIdx.x; n < N; n += tpr) s += fast_ex2((Elem<T>::load(xr + n) - m) * kLog2e);
         s = group_reduce<false>(s, tpr, red);
         const float inv = 1.0f / s;
         for (long long n = threadIdx.x; n < N; n += tpr)
-            Elem<T>::store(yr + n, exp2f((Elem<T>::load(xr + n) - m) * kLog2e) * inv);
+            Elem<T>::store(yr + n, fast_ex2((Elem<T>::load(xr + n) - m) * kLog2e) * inv);
     } else {
         float mean = 0.f;
         if (NORM == KF_NORM_LAYERNORM) {

@@ -405,7 +405,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
                             const bool full = (c + 1) * 32 <= ncols;
 #pragma unroll
                             for (int e = 0; e < 32; ++e) {
-                                a[e] = exp2f(fmaf(a[e], kLog2e, -ms));
+                                a[e] = fast_ex2(fmaf(a[e], kLog2e, -ms));
                                 if (full || c * 32 + e < ncols) l4[e & 3] += a[e];
                             }
 #pragma unroll
@@ -501,7 +501,7 @@ tc_rownorm_finish_kernel(__nv_bfloat16* Y, long long ldy, int M, int N, int nsub
         float l = 0.f;
         for (int s = gt; s < nsub; s += gsize) {
             const float4 q = pr[s];
-            const float f = exp2f((q.x - m) * kLog2e);
+            const float f = fast_ex2((q.x - m) * kLog2e);
             coef[s] = make_float2(f, 0.f);
             l = fmaf(q.y, f, l);
         }
