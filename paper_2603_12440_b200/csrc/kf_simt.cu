@@ -44,28 +44,40 @@ simt_rows_kernel(const T* __restrict__ X, long long ldx, const T* __restrict__ W
 #pragma unroll
         for (int j = 0; j < NPT; ++j) acc[i][j] = 0.f;
 
-    for (int k0 = 0; k0 < K; k0 += kSlabK) {
-        __syncthreads();
-        for (int e = t; e < BM * kSlabK; e += kThreads) {
-            const int i = e / kSlabK, kk = e % kSlabK;
-            xs[i][kk] = (m0 + i < M && k0 + kk < K) ? Elem<T>::load(X + (long long)(m0 + i) * ldx + k0 + kk) : 0.f;
+    // Software pipeline over (k0, j) steps: the global loads of the next step are issued before the
+    // FMAs of the current one, so their latency hides behind the arithmetic and the barriers.
+    static_assert(BM * kSlabK <= kThreads, "one X element per thread and step");
+    auto load_w = [&](float (&tmp)[32], int k0, int j) {
+#pragma unroll
+        for (int u = 0; u < 32; ++u) {
+            const int n = j * kThreads + u * (kThreads / 32) + warp;      // a warp reads one W row per step (coalesced)
+            tmp[u] = (n < N && k0 + lane < K) ? Elem<T>::load(W + (long long)n * ldw + k0 + lane) : 0.f;
         }
+    };
+    auto load_x = [&](int k0) -> float {
+        const int i = t / kSlabK, kk = t % kSlabK;
+        return (t < BM * kSlabK && m0 + i < M && k0 + kk < K) ? Elem<T>::load(X + (long long)(m0 + i) * ldx + k0 + kk) : 0.f;
+    };
+    float tmp[32];
+    float xv = 0.f;
+    if (K > 0) {
+        load_w(tmp, 0, 0);
+        xv = load_x(0);
+    }
+    for (int k0 = 0; k0 < K; k0 += kSlabK) {
 #pragma unroll
         for (int j = 0; j < NPT; ++j) {
-            if (j > 0) __syncthreads();
-            // slab j: W rows j*256 .. j*256+255, k0 .. k0+31; a warp reads one row per step (coalesced)
-            // 32 rows per warp; the loads are independent, so all are issued before the first store
-            {
-                float tmp[32];
+            __syncthreads();                               // the previous step's FMAs are done with ws / xs
 #pragma unroll
-                for (int u = 0; u < 32; ++u) {
-                    const int n = j * kThreads + u * (kThreads / 32) + warp;
-                    tmp[u] = (n < N && k0 + lane < K) ? Elem<T>::load(W + (long long)n * ldw + k0 + lane) : 0.f;
-                }
-#pragma unroll
-                for (int u = 0; u < 32; ++u) ws[u * (kThreads / 32) + warp][lane] = tmp[u];
-            }
+            for (int u = 0; u < 32; ++u) ws[u * (kThreads / 32) + warp][lane] = tmp[u];
+            if (j == 0 && t < BM * kSlabK) xs[t / kSlabK][t % kSlabK] = xv;
             __syncthreads();
+            if (j + 1 < NPT) {
+                load_w(tmp, k0, j + 1);
+            } else if (k0 + kSlabK < K) {
+                load_w(tmp, k0 + kSlabK, 0);
+                xv = load_x(k0 + kSlabK);
+            }
 #pragma unroll
             for (int kk = 0; kk < kSlabK; ++kk) {
                 const float w = ws[t][kk];
