@@ -283,3 +283,37 @@ def test_tc32_matches_oracle_under_the_fp32_gate(kf, norm):
     assert cfg["kernel"] == 4 and cfg["row_scheme"] == (0 if norm == "none" else 4)
     r = assert_parity(run(kf, p), oracle_of(p), "f32", f"tc32 {norm}")
     assert r["max_abs"] < 2e-5
+
+
+def test_calls_on_a_side_stream_and_growing_workspace(kf):
+    """The library launches on the stream it is given: results computed on a side stream, with the
+    binding's cached workspace growing between calls of different sizes, match the oracle."""
+    side = torch.cuda.Stream()
+    small = make("bf16", 130, 264, 72, seed=41, act="relu", norm="softmax")
+    large = make("bf16", 520, 4104, 136, seed=42, act="silu", norm="layernorm", res=True)
+    outs = []
+    with torch.cuda.stream(side):
+        for p in (small, large, small):
+            d = problem_to_device(p)
+            outs.append((p, kf.linear_epilogue_rownorm(d["X"], d["W"], d["bias"], p.act, p.scale, d["residual"],
+                                                       p.norm, d["gamma"], d["beta"], p.eps)))
+        kf.check_device_status()
+    side.synchronize()
+    for p, y in outs:
+        assert_parity(to_f64(y), oracle_of(p), "bf16", f"side stream {p.M}x{p.N}")
+
+
+def test_noalloc_form_rejects_a_large_fp32_call(kf):
+    # the tensor-core fp32 path needs split copies of X and W: far beyond the built-in scratch
+    x = torch.zeros(8192, 4096, device="cuda")
+    w = torch.zeros(4096, 4096, device="cuda")
+    out = torch.empty(8192, 4096, device="cuda")
+    with pytest.raises(kf.KfError) as e:
+        kf.linear_epilogue_rownorm_noalloc(x, w, out)
+    assert e.value.status == 7
+    # while a small fp32 call needs no scratch beyond the status block and goes through
+    p = inputs.config(1)
+    d = problem_to_device(p)
+    y = torch.empty(p.M, p.N, device="cuda")
+    kf.linear_epilogue_rownorm_noalloc(d["X"], d["W"], y, d["bias"], p.act, p.scale, None, p.norm, wait=True)
+    assert_parity(to_f64(y), oracle_of(p), "f32", "noalloc C1")
