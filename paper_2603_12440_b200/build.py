@@ -13,8 +13,9 @@ from pathlib import Path
 PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libkf.so"
-SOURCES = ["kf_api.cu", "kf_row.cu", "kf_simt.cu", "kf_tc.cu", "kf_tc32.cu"]
-HEADERS = ["kf_common.cuh", "kf_tc.cuh", "kf_tc_ptx.cuh", "../../include/kf.h"]
+SOURCES = ["kf_api.cu", "kf_row.cu", "kf_simt.cu", "kf_tc.cu", "kf_tc_spec_none.cu", "kf_tc_spec_softmax.cu",
+           "kf_tc_spec_layernorm.cu", "kf_tc_spec_rmsnorm.cu", "kf_tc32.cu"]
+HEADERS = ["kf_common.cuh", "kf_tc.cuh", "kf_tc_ptx.cuh", "kf_tc_kernel.cuh", "../../include/kf.h"]
 
 
 def nvcc_path() -> str:

@@ -1,0 +1,618 @@
+// bf16 linear + epilogue (+ split-N row-norm) on the Blackwell tensor cores: tcgen05.mma with the
+// accumulator in TMEM, operands staged by TMA into 128B-swizzled shared memory, written for
+// sm_100a only.
+//
+// One persistent CTA per SM walks output tiles of BM x BN = 128 x 256 (row-block major, so the
+// N-tiles of one row block run side by side); with CTA pairs (CG 2) a work unit is 256 x 256.
+// Twelve warps in three warpgroups:
+//   warp 0       TMA producer: X tile [128 x 64] and W tile [256 / CG x 64] per k-block into the ring
+//                (6 stages of 32 KiB for CG 2, 4 stages of 48 KiB for CG 1)
+//   warp 1       allocates TMEM (512 columns = two accumulators) and issues tcgen05.mma
+//   warps 2..3   idle: they fill warpgroup 0, which gives most of its registers away
+//   warps 4..11  epilogue: two warps per TMEM lane quarter, 128 columns each (thread = output row)
+// After set-up warpgroup 0 drops to 40 registers per thread and the epilogue warpgroups rise to 232
+// (setmaxnreg).  An epilogue thread reads its 128 accumulator columns into registers with four
+// tcgen05.ld and hands the accumulator back to the MMA warp at once, so the main loop of the next
+// units never waits for epilogue math; bias (staged as fp32 in shared memory) / activation / scale /
+// residual run in fp32 in registers, then the 16-bit values go through a per-warp, double-buffered
+// 32 x 64-byte staging block (64-byte swizzle, conflict-free) and leave as TMA stores, which also
+// clip the rows and columns beyond Y.
+//
+// Row-norm (split-N): a row of N outputs spans N/128 sub-tiles owned by different warps and CTAs.
+// With the sub-tile row in registers the thread gathers its statistics, then turns the values into
+// a 16-bit intermediate stored in Y -- softmax: bf16 exp(a - tile max); LayerNorm / RMSNorm: fp16
+// (a - tile shift) * 2^-e with a per-row, per-tile power-of-two block scale, so the intermediate
+// carries 11 significant bits relative to the largest deviation of the tile row.  The per-row
+// partial {shift or max, sum, sum of squares, 2^e} goes to the workspace; the finishing kernel
+// merges the partials of a row (online-softmax rescaling / Chan's merge) and rescales in place.
+//
+// Every wait on an mbarrier is bounded: when it gives up it records KF_ERR_TIMEOUT in the
+// workspace status word, raises a CTA-wide abort flag and the CTA drains and exits.
+//
+// This header holds the kernel template; kf_tc.cu instantiates the generic form (row-norm and
+// activation read from the parameters, timing switches honoured) and kf_tc_spec*.cu the forms
+// with both fixed at compile time, whose straight-line epilogue is a fraction of the size: the
+// epilogue code is fully unrolled over the 128 columns a thread owns, and its instruction
+// footprint, not its arithmetic, is what the generic form pays for.
+#pragma once
+#include <cuda.h>
+#include <cuda_fp16.h>
+
+#include <mutex>
+
+#include "kf_tc.cuh"
+#include "kf_tc_ptx.cuh"
+
+namespace kf {
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64, UMMA_K = 16;
+constexpr int kMaxStages = 6;
+constexpr int kEpiWarps = 8;                           // two per TMEM lane quarter, 128 columns each
+constexpr int kSub = BN / 2;                           // columns per epilogue warp = statistics sub-tile
+constexpr int kRoleWarps = 4;                          // warpgroup 0: TMA producer, MMA issuer, two idle warps
+constexpr int kThreads = 32 * (kRoleWarps + kEpiWarps);
+// Registers: 384 threads start with 168 each; warpgroup 0 keeps 40 and the epilogue warpgroups take
+// 232 (4*40 + 8*232 = 12*168), which the fully unrolled 32-column epilogue needs to overlap its
+// independent element chains instead of running them one after the other.
+constexpr int kRegsLaunch = 168, kRegsRole = 40, kRegsEpi = 232;
+static_assert(kRoleWarps * kRegsRole + kEpiWarps * kRegsEpi <= (kRoleWarps + kEpiWarps) * kRegsLaunch, "register pool");
+constexpr int kTmemCols = 512;                         // two fp32 accumulators of BN columns
+constexpr uint32_t kABytes = BM * BK * 2;              // 16 KiB
+// CG = CTAs per MMA.  CG 1: a CTA stages the whole 256-row W tile (32 KiB, 4 stages).  CG 2: the two
+// CTAs of a cluster stage 128 rows of W each (16 KiB, 6 stages) and one tcgen05.mma.cta_group::2
+// of M = 256 reads both halves, which halves the shared-memory traffic per flop.
+template <int CG> struct Cfg {
+    static constexpr int kStages = CG == 2 ? 6 : 4;
+    static constexpr uint32_t kBRows = BN / CG;
+    static constexpr uint32_t kBBytes = kBRows * BK * 2;
+    static constexpr uint32_t kStageBytes = kABytes + kBBytes;
+    static constexpr uint32_t kSmemB = kStages * kABytes;
+    static_assert(kStages * kStageBytes == 192 * 1024, "operand ring is 192 KiB in both modes");
+};
+constexpr uint32_t kSmemA = 0;
+// store staging behind the operand ring: per epilogue warp two buffers of 32 rows x 64 bytes (one
+// 32-column chunk of its 32 rows, 64-byte swizzled), written by the warp and drained by TMA stores
+constexpr uint32_t kSmemStage = 192 * 1024;
+constexpr uint32_t kStageBufBytes = 32 * 64;
+constexpr uint32_t kSmemBias = kSmemStage + kEpiWarps * 2 * kStageBufBytes;   // 2 x BN floats (double buffered)
+constexpr uint32_t kSmemBar = kSmemBias + 2 * BN * 4;
+constexpr uint32_t kNumBars = 2 * kMaxStages + 6;         // ring full/empty, accumulator full/empty, bias ready
+constexpr uint32_t kSmemTmemPtr = kSmemBar + kNumBars * 8;
+constexpr uint32_t kSmemAbort = kSmemTmemPtr + 8;      // abort flag (4 B, 8-byte aligned), then the wait limit (8 B)
+constexpr uint32_t kSmemAlloc = kSmemAbort + 16;
+static_assert(kSmemAlloc <= 232448, "exceeds the 227 KiB per-CTA shared memory of sm_100");
+
+// instruction descriptor: D fp32, A and B bf16, both K-major, M = 128 * CG, N = 256
+template <int CG>
+constexpr uint32_t kIdesc =
+    (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((BM * CG) >> 4) << 24);
+
+struct TcParams {
+    int M, N, K;
+    int tiles_m, tiles_n;
+    int nsub;                   // statistics sub-tiles per row = ceil(N / 128)
+    const __nv_bfloat16* bias;
+    const __nv_bfloat16* residual;
+    long long ldr;
+    int act;
+    float scale;
+    int norm;
+    float4* partials;           // [tiles_m * 128 rows][nsub] when norm != NONE
+    uint32_t* status;
+    __nv_bfloat16* Y;           // output (or 16-bit intermediate), row pitch ldy
+    long long ldy;
+    int debug;                  // generic form only; timing experiments (results are wrong): 1 no TMA loads, 2 no MMAs,
+                                // 4 no epilogue work, 8 no stores, 16 no TMEM loads, 32 no activation, 64 no residual,
+                                // 256 a longer epilogue; 128 = register stores instead of TMA stores (results right);
+                                // 512 = the producer never signals, so every wait runs into its limit (time-out test);
+                                // 1024 = cycle counters of the roles added into words 8..19 of the status block
+    long long timeout_cycles;   // limit of every bounded wait
+};
+
+// element-wise epilogue on 32 consecutive columns of one row, fast-math forms (bf16 output).
+// bias32: the 32 bias values as fp32 in shared memory (or nullptr); col0 = global column of a[0];
+// 8-column vectors at or beyond N are not read from the residual.
+__device__ __forceinline__ void epilogue32(float (&a)[32], const TcParams& p, const int act, const int debug,
+                                           const float* bias32, long long row, int col0, bool row_ok) {
+    // the residual comes from global memory (often DRAM): issue its loads first, use them last
+    const bool has_res = p.residual && row_ok && !(debug & 64);
+    uint4 rv[4];
+    if (has_res) {
+        const int left = p.N - col0;
+        const uint4* rp = reinterpret_cast<const uint4*>(p.residual + row * p.ldr + col0);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) rv[q] = (q * 8 < left) ? __ldg(rp + q) : make_uint4(0, 0, 0, 0);
+    }
+    if (bias32) {
+        const float4* bp = reinterpret_cast<const float4*>(bias32);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const float4 b = bp[q];
+            a[q * 4 + 0] += b.x; a[q * 4 + 1] += b.y; a[q * 4 + 2] += b.z; a[q * 4 + 3] += b.w;
+        }
+    }
+    if (act != KF_ACT_NONE && !(debug & 32)) {
+        switch (act) {
+        case KF_ACT_GELU_ERF:
+#pragma unroll
+            for (int e = 0; e < 32; ++e) a[e] = apply_act<false>(KF_ACT_GELU_ERF, a[e]);
+            break;
+        case KF_ACT_GELU_TANH:
+#pragma unroll
+            for (int e = 0; e < 32; ++e) a[e] = apply_act<false>(KF_ACT_GELU_TANH, a[e]);
+            break;
+        case KF_ACT_SILU:
+#pragma unroll
+            for (int e = 0; e < 32; ++e) a[e] = apply_act<false>(KF_ACT_SILU, a[e]);
+            break;
+        case KF_ACT_RELU:
+#pragma unroll
+            for (int e = 0; e < 32; ++e) a[e] = fmaxf(a[e], 0.f);
+            break;
+        default:
+#pragma unroll
+            for (int e = 0; e < 32; ++e) a[e] = apply_act<false>(KF_ACT_SIGMOID, a[e]);
+            break;
+        }
+    }
+    if (p.scale != 1.0f) {
+#pragma unroll
+        for (int e = 0; e < 32; ++e) a[e] *= p.scale;
+    }
+    if (has_res) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            float r[8];
+            unpack<__nv_bfloat16>(rv[q], r);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) a[q * 8 + e] += r[e];
+        }
+    }
+}
+
+// one thread writes its 32 packed 16-bit values (64 contiguous bytes of its output row); 8-column
+// vectors at or beyond the valid columns are skipped
+__device__ __forceinline__ void store_row32(__nv_bfloat16* dst, const uint32_t (&w)[16], int valid_cols) {
+    uint4* d = reinterpret_cast<uint4*>(dst);
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+        if (j * 8 < valid_cols) d[j] = make_uint4(w[j * 4 + 0], w[j * 4 + 1], w[j * 4 + 2], w[j * 4 + 3]);
+}
+
+// NORM / ACT: the row-norm and activation compiled in, or -1 for the generic form that reads both
+// from the parameters and honours the timing switches (p.debug).
+template <int CG, int NORM, int ACT>
+__global__ void __launch_bounds__(kThreads, 1)
+tc_linear_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW,
+                 const __grid_constant__ CUtensorMap tmY, const TcParams p) {
+    static_assert((NORM < 0) == (ACT < 0), "generic in both or in neither");
+    constexpr bool kGeneric = NORM < 0;
+    const int norm = kGeneric ? p.norm : NORM;
+    const int act = kGeneric ? p.act : ACT;
+    const int debug = kGeneric ? p.debug : 0;
+    // cycle counters of the generic form (debug bit 1024): how long the MMA thread waits for operands
+    // and for a free accumulator, how long the epilogue waits, holds the accumulator and works
+    auto tick = [&]() -> long long { return kGeneric ? clock64() : 0ll; };
+    using C = Cfg<CG>;
+    constexpr int kStages = C::kStages;
+    constexpr uint32_t kSmemB = C::kSmemB, kBBytes = C::kBBytes;
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const uint32_t base = smem_u32(smem_raw);
+    if (base & 1023u) {                                 // swizzled tiles need a 1024-byte aligned base
+        if (threadIdx.x == 0 && atomicCAS(p.status, 0u, (uint32_t)KF_ERR_CUDA) == 0u) p.status[1] = 0x900u;
+        return;                                         // (same in both CTAs of a pair: the layout is identical)
+    }
+    const uint32_t rank = CG == 2 ? cluster_ctarank() : 0u;       // rank 0 of a pair issues the MMAs
+    const int unit = CG == 2 ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+    const int num_units = CG == 2 ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+    const uint32_t bar0 = base + kSmemBar;
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
+    auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kStages + a); };
+    auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kStages + 2 + a); };
+    auto bias_bar = [&](int b) { return bar0 + 8u * (2 * kStages + 4 + b); };
+    volatile uint32_t* tmem_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + kSmemTmemPtr);
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem_raw + kSmemAbort);
+    float* bias_smem = reinterpret_cast<float*>(smem_raw + kSmemBias);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // a work unit is a BM*CG x BN block of the output: one tile, or the two row-adjacent tiles of a pair
+    const int units_m = (p.tiles_m + CG - 1) / CG;
+    const int num_tiles = units_m * p.tiles_n;
+    const int kblocks = (p.K + BK - 1) / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(tfull_bar(a), 1);
+            mbar_init(tempty_bar(a), kEpiWarps * CG);   // the leader's collects the epilogue warps of both CTAs
+            mbar_init(bias_bar(a), kEpiWarps);
+        }
+        *abort_flag = 0;
+        *reinterpret_cast<volatile long long*>(smem_raw + kSmemAbort + 8) = p.timeout_cycles;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        if (CG == 2) {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(base + kSmemTmemPtr),
+                         "r"((uint32_t)kTmemCols)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(base + kSmemTmemPtr),
+                         "r"((uint32_t)kTmemCols)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (CG == 2) cluster_sync_all();                    // the peer's barriers exist before anyone signals them
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_ptr;
+
+    if (warp < kRoleWarps) {
+      reg_dealloc<kRegsRole>();
+      if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            bool ok = true;
+            for (int tile = unit; tile < num_tiles && ok; tile += num_units) {
+                if (debug & 512) break;                  // time-out test: nothing is ever loaded or signalled
+                const int mb = (tile / p.tiles_n) * CG + (int)rank, nb = tile % p.tiles_n;
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    if (!mbar_wait_inl(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 0x100u + stage)) { ok = false; break; }
+                    if (debug & 1) {
+                        if (rank == 0) mbar_arrive(full_bar(stage));
+                    } else if (CG == 2) {
+                        // both CTAs' copies complete on the leader's barrier, which expects the bytes of both
+                        if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2 * C::kStageBytes);
+                        const uint32_t lead_bar = map_to_cta(full_bar(stage), 0);
+                        tma_load_2d_pair(base + kSmemA + stage * kABytes, &tmX, lead_bar, kb * BK, mb * BM);
+                        tma_load_2d_pair(base + kSmemB + stage * kBBytes, &tmW, lead_bar, kb * BK,
+                                         nb * BN + (int)(rank * C::kBRows));
+                    } else {
+                        mbar_arrive_expect_tx(full_bar(stage), C::kStageBytes);
+                        tma_load_2d(base + kSmemA + stage * kABytes, &tmX, full_bar(stage), kb * BK, mb * BM);
+                        tma_load_2d(base + kSmemB + stage * kBBytes, &tmW, full_bar(stage), kb * BK, nb * BN);
+                    }
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+      } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0 && rank == 0) {
+            uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
+            bool ok = true;
+            long long tw_acc = 0, tw_full = 0;
+            const long long tm0 = tick();
+            for (int tile = unit; tile < num_tiles && ok; tile += num_units) {
+                const long long ta = tick();
+                if (!mbar_wait_inl(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status, 0x200u + acc)) { ok = false; break; }
+                tw_acc += tick() - ta;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * BN;
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    const long long tf = tick();
+                    if (!mbar_wait_inl(full_bar(stage), phase, abort_flag, p.status, 0x300u + stage)) { ok = false; break; }
+                    tw_full += tick() - tf;
+                    tc_fence_after();
+                    const uint32_t a_addr = base + kSmemA + stage * kABytes;
+                    const uint32_t b_addr = base + kSmemB + stage * kBBytes;
+#pragma unroll
+                    for (int k = 0; k < BK / UMMA_K; ++k) {
+                        if (debug & 2) break;
+                        const uint64_t ad = smem_desc_sw128(a_addr + k * UMMA_K * 2);
+                        const uint64_t bd = smem_desc_sw128(b_addr + k * UMMA_K * 2);
+                        if (CG == 2) tc_mma_bf16_pair(d_tmem, ad, bd, kIdesc<2>, (kb | k) != 0 ? 1u : 0u);
+                        else tc_mma_bf16(d_tmem, ad, bd, kIdesc<1>, (kb | k) != 0 ? 1u : 0u);
+                    }
+                    // stage reusable (in both CTAs of a pair) once these MMAs have read it
+                    if (CG == 2) {
+                        tc_commit_pair(empty_bar(stage));
+                        tc_commit_pair(map_to_cta(empty_bar(stage), 1));
+                    } else {
+                        tc_commit(empty_bar(stage));
+                    }
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                // accumulator complete: each CTA's epilogue reads its own 128 rows
+                if (CG == 2) {
+                    tc_commit_pair(tfull_bar(acc));
+                    tc_commit_pair(map_to_cta(tfull_bar(acc), 1));
+                } else {
+                    tc_commit(tfull_bar(acc));
+                }
+                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            }
+            if (debug & 1024) {
+                unsigned long long* t64 = reinterpret_cast<unsigned long long*>(p.status);
+                atomicAdd(t64 + 6, (unsigned long long)tw_acc);
+                atomicAdd(t64 + 7, (unsigned long long)tw_full);
+                atomicAdd(t64 + 8, (unsigned long long)(tick() - tm0));
+            }
+        }
+      }
+    } else {
+        reg_alloc<kRegsEpi>();
+        // ------------------------------------------------------------------ epilogue warps
+        const int q = warp & 3;                            // TMEM lane quarter this warp may access
+        const int half = (warp - kRoleWarps) >> 2;         // which 128 columns of the tile
+        const int et = threadIdx.x - 32 * kRoleWarps;      // 0..255 among the epilogue threads
+        uint32_t acc = 0, acc_phase = 0, it = 0, nstore = 0;
+        const uint32_t stage_base = base + kSmemStage + (uint32_t)(warp - kRoleWarps) * 2u * kStageBufBytes;
+        bool ok = true;
+        long long te_wait = 0, te_work = 0, te_s1 = 0;
+        for (int tile = unit; tile < num_tiles && ok; tile += num_units, ++it) {
+            const long long te0 = tick();
+            const int mb = (tile / p.tiles_n) * CG + (int)rank, nb = tile % p.tiles_n;
+            const int m0 = mb * BM, n0 = nb * BN;
+            const int cb = half * kSub;                    // first tile column of this warp
+            const long long row = (long long)m0 + q * 32 + lane;
+            const bool row_ok = row < p.M;
+            const int ncols = max(0, min(kSub, p.N - n0 - cb));     // valid columns of this warp (multiple of 8)
+            const int nchunks = (debug & 4) ? 0 : (ncols + 31) >> 5;
+
+            // bias of the tile as fp32 in shared memory, double buffered across tiles
+            float* bias_t = nullptr;
+            if (p.bias) {
+                bias_t = bias_smem + (it & 1u) * BN;
+                bias_t[et] = (n0 + et < p.N) ? __bfloat162float(p.bias[n0 + et]) : 0.f;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bias_bar(it & 1u));        // release: this warp's 32 values are written
+                if (!mbar_wait_inl(bias_bar(it & 1u), (it >> 1) & 1u, abort_flag, p.status, 0x500u)) { ok = false; break; }
+                bias_t += cb;
+            }
+            if (!mbar_wait_inl(tfull_bar(acc), acc_phase, abort_flag, p.status, 0x400u + acc)) { ok = false; break; }
+            tc_fence_after();
+            const long long te1 = tick();
+            te_wait += te1 - te0;
+            const uint32_t t_row = tmem_base + acc * BN + cb + ((uint32_t)(q * 32) << 16);
+
+            // the thread's 128 accumulator columns go to registers in one go and the accumulator is handed
+            // back to the MMA warp before any math: the epilogue then overlaps the next main loops freely
+            uint32_t v[kSub / 32][32];
+            if (!(debug & 16)) {
+#pragma unroll
+                for (int c = 0; c < kSub / 32; ++c)
+                    if (c < nchunks) tc_ld32_issue(t_row + c * 32, v[c]);
+#pragma unroll
+                for (int c = 0; c < kSub / 32; ++c) tc_ld_wait(v[c]);
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+                if (CG == 2 && rank != 0) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
+                else mbar_arrive(tempty_bar(acc));
+            }
+            te_s1 += tick() - te1;
+
+            // element-wise epilogue in place, per-row statistics of the sub-tile (4 independent accumulators each)
+            float st_shift = 0.f, st_s1 = 0.f, st_s2 = 0.f, st_scale = 1.f, mult = 1.f;
+            float s1[4] = {0.f, 0.f, 0.f, 0.f}, s2[4] = {0.f, 0.f, 0.f, 0.f};
+            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY}, am[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int c = 0; c < kSub / 32; ++c) {
+                if (c < nchunks) {
+                    float a[32];
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) a[e] = __uint_as_float(v[c][e]);
+                    epilogue32(a, p, act, debug, bias_t ? bias_t + c * 32 : nullptr, row, n0 + cb + c * 32, row_ok);
+                    const bool full = (c + 1) * 32 <= ncols;
+                    if (norm == KF_NORM_SOFTMAX) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e)
+                            if (full || c * 32 + e < ncols) mx[e & 3] = fmaxf(mx[e & 3], a[e]);
+                    } else if (norm != KF_NORM_NONE) {
+                        if (norm == KF_NORM_LAYERNORM) {
+                            if (c == 0) st_shift = a[0];
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) a[e] -= st_shift;
+                        }
+#pragma unroll
+                        for (int e = 0; e < 32; ++e)
+                            if (full || c * 32 + e < ncols) {
+                                s1[e & 3] += a[e];
+                                s2[e & 3] = fmaf(a[e], a[e], s2[e & 3]);
+                                am[e & 3] = fmaxf(am[e & 3], fabsf(a[e]));
+                            }
+                    }
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) v[c][e] = __float_as_uint(a[e]);
+                }
+            }
+            if (norm == KF_NORM_SOFTMAX) {
+                st_shift = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+            } else if (norm != KF_NORM_NONE) {
+                st_s1 = (s1[0] + s1[1]) + (s1[2] + s1[3]);
+                st_s2 = (s2[0] + s2[1]) + (s2[2] + s2[3]);
+                const float amax = fmaxf(fmaxf(am[0], am[1]), fmaxf(am[2], am[3]));
+                // power-of-two block scale: stored fp16 values lie in (-2, 2)
+                uint32_t eb = (__float_as_uint(amax) >> 23) & 0xFFu;
+                eb = min(max(eb, 1u), 253u);
+                st_scale = __uint_as_float(eb << 23);
+                mult = __uint_as_float((254u - eb) << 23);
+            }
+            // 16-bit pack and store: the result (no row-norm) or the intermediate the finishing kernel rescales
+            {
+                float l4[4] = {0.f, 0.f, 0.f, 0.f};
+                const float ms = st_shift * kLog2e;
+#pragma unroll
+                for (int c = 0; c < kSub / 32; ++c) {
+                    if (c < nchunks) {
+                        float a[32];
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) a[e] = __uint_as_float(v[c][e]);
+                        uint32_t w[16];
+                        if (norm == KF_NORM_NONE) {
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) w[e] = pack_bf16(a[2 * e], a[2 * e + 1]);
+                        } else if (norm == KF_NORM_SOFTMAX) {
+                            const bool full = (c + 1) * 32 <= ncols;
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) {
+                                a[e] = fast_ex2(fmaf(a[e], kLog2e, -ms));
+                                if (full || c * 32 + e < ncols) l4[e & 3] += a[e];
+                            }
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) w[e] = pack_bf16(a[2 * e], a[2 * e + 1]);
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) w[e] = pack_f16(a[2 * e] * mult, a[2 * e + 1] * mult);
+                        }
+                        if (debug & 128) {
+                            if (row_ok && !(debug & 8))
+                                store_row32(p.Y + row * p.ldy + n0 + cb + c * 32, w, ncols - c * 32);
+                        } else if (!(debug & 8)) {
+                            // the warp's 32 rows x 64 bytes go to its staging buffer (16-byte pieces XOR-swizzled
+                            // with bits 1-2 of the row, the 64-byte TMA pattern: conflict-free), then one TMA
+                            // store writes the block; rows and columns outside Y are clipped by the copy
+                            const uint32_t sbuf = stage_base + (uint32_t)(nstore & 1u) * kStageBufBytes;
+                            if (nstore >= 2) {              // the store that last read this buffer has drained it
+                                if (lane == 0) tma_store_wait_read<1>();
+                                __syncwarp();
+                            }
+                            const uint32_t srow = sbuf + (uint32_t)lane * 64u;
+                            const uint32_t sw = ((uint32_t)lane >> 1) & 3u;
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+                                st_shared_v4(srow + ((((uint32_t)j) ^ sw) << 4), w[j * 4 + 0], w[j * 4 + 1], w[j * 4 + 2],
+                                             w[j * 4 + 3]);
+                            fence_async_smem();
+                            __syncwarp();
+                            if (lane == 0) {
+                                tma_store_2d(&tmY, sbuf, n0 + cb + c * 32, m0 + q * 32);
+                                tma_store_commit();
+                            }
+                            ++nstore;
+                        }
+                    }
+                }
+                if (norm == KF_NORM_SOFTMAX) st_s1 = (l4[0] + l4[1]) + (l4[2] + l4[3]);
+            }
+            if (debug & 256) {                            // timing experiment: a 5 us longer epilogue
+                const long long t0 = clock64();
+                while (clock64() - t0 < 10000) {}
+            }
+            if (norm != KF_NORM_NONE && row_ok && nchunks > 0)
+                p.partials[((size_t)mb * BM + q * 32 + lane) * p.nsub + (nb * 2 + half)] =
+                    make_float4(st_shift, st_s1, st_s2, st_scale);
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            te_work += tick() - te1;
+        }
+        if (lane == 0) tma_store_wait_all<0>();              // the staging buffers are read, Y is written
+        if ((debug & 1024) && warp == kRoleWarps && lane == 0) {
+            unsigned long long* t64 = reinterpret_cast<unsigned long long*>(p.status);
+            atomicAdd(t64 + 4, (unsigned long long)te_wait);
+            atomicAdd(t64 + 5, (unsigned long long)te_work);
+            atomicAdd(t64 + 9, (unsigned long long)te_s1);
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (CG == 2) cluster_sync_all();                    // neither CTA leaves while the peer may still signal it
+    if (warp == 1) {
+        if (*abort_flag) {
+            // give copies and MMAs in flight a bounded time to land before TMEM goes away
+            for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+        }
+        tc_fence_after();
+        if (CG == 2)
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                         "r"((uint32_t)kTmemCols)
+                         : "memory");
+        else
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                         "r"((uint32_t)kTmemCols)
+                         : "memory");
+    }
+}
+
+// ------------------------------------------------------------------------------ finishing kernel
+// WPR warps per row (1, 2, 4 or 8; a CTA of 8 warps holds 8 / WPR rows): merge the row's per-sub-tile
+// partials (warp shuffles + one shared-memory hop across the row's warps), then rescale the 16-bit
+// intermediates of the row in place with up to 8 independent 128-bit accesses in flight per lane.
+
+// One instantiation: opt in to the large dynamic shared memory and check the register allowance once
+// per device, then launch on `st` (as clusters of two for CG 2).
+template <int CG, int NORM, int ACT>
+kf_status tc_launch_instance(int grid, cudaStream_t st, const CUtensorMap& tmX, const CUtensorMap& tmW,
+                             const CUtensorMap& tmY, const TcParams& p) {
+    auto kernel = tc_linear_kernel<CG, NORM, ACT>;
+    {
+        static std::mutex mu;
+        static bool done[64] = {};
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return KF_ERR_CUDA;
+        std::lock_guard<std::mutex> lock(mu);
+        if (!done[dev]) {
+            if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemAlloc) != cudaSuccess)
+                return KF_ERR_CUDA;
+            // the in-kernel register re-allocation assumes the launch allowance it was written for: a build
+            // with fewer registers per thread would leave the epilogue warps waiting for registers that
+            // no warp gives back, so such a build is refused here rather than launched
+            cudaFuncAttributes fa;
+            if (cudaFuncGetAttributes(&fa, kernel) != cudaSuccess || fa.numRegs < kRegsLaunch) return KF_ERR_CUDA;
+            done[dev] = true;
+        }
+    }
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3((unsigned)grid);
+    lc.blockDim = dim3(kThreads);
+    lc.dynamicSmemBytes = kSmemAlloc;
+    lc.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = CG;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    lc.attrs = at;
+    lc.numAttrs = 1;
+    if (cudaLaunchKernelEx(&lc, kernel, tmX, tmW, tmY, p) != cudaSuccess) {
+        cudaGetLastError();
+        return KF_ERR_CUDA;
+    }
+    return KF_OK;
+}
+
+// the six activations of one row-norm (CTA pairs)
+template <int NORM>
+kf_status tc_launch_norm(int act, int grid, cudaStream_t st, const CUtensorMap& tmX, const CUtensorMap& tmW,
+                         const CUtensorMap& tmY, const TcParams& p) {
+    switch (act) {
+    case KF_ACT_NONE: return tc_launch_instance<2, NORM, KF_ACT_NONE>(grid, st, tmX, tmW, tmY, p);
+    case KF_ACT_GELU_ERF: return tc_launch_instance<2, NORM, KF_ACT_GELU_ERF>(grid, st, tmX, tmW, tmY, p);
+    case KF_ACT_GELU_TANH: return tc_launch_instance<2, NORM, KF_ACT_GELU_TANH>(grid, st, tmX, tmW, tmY, p);
+    case KF_ACT_SILU: return tc_launch_instance<2, NORM, KF_ACT_SILU>(grid, st, tmX, tmW, tmY, p);
+    case KF_ACT_RELU: return tc_launch_instance<2, NORM, KF_ACT_RELU>(grid, st, tmX, tmW, tmY, p);
+    case KF_ACT_SIGMOID: return tc_launch_instance<2, NORM, KF_ACT_SIGMOID>(grid, st, tmX, tmW, tmY, p);
+    default: return KF_ERR_INVALID_ARG;
+    }
+}
+
+}  // namespace
+
+// specialised CTA-pair kernels, one translation unit per row-norm (kf_tc_spec*.cu)
+struct TcLaunchArgs {
+    int grid;
+    cudaStream_t st;
+    const CUtensorMap* tmX;
+    const CUtensorMap* tmW;
+    const CUtensorMap* tmY;
+    const void* params;         // TcParams of the calling translation unit (same definition)
+};
+kf_status tc_launch_spec_none(int act, const TcLaunchArgs& a);
+kf_status tc_launch_spec_softmax(int act, const TcLaunchArgs& a);
+kf_status tc_launch_spec_layernorm(int act, const TcLaunchArgs& a);
+kf_status tc_launch_spec_rmsnorm(int act, const TcLaunchArgs& a);
+
+}  // namespace kf

@@ -37,8 +37,8 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 }
 
 // bounded wait: false = gave up (status recorded, abort raised) or another role aborted
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                            uint32_t* status, uint32_t code) {
+__device__ __forceinline__ bool mbar_wait_spin(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                               uint32_t* status, uint32_t code) {
     const long long limit = *reinterpret_cast<volatile long long*>(const_cast<uint32_t*>(abort_flag) + 2);
     const long long t0 = clock64();
     uint32_t spins = 0;
@@ -55,10 +55,28 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volat
     }
     return true;
 }
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                            uint32_t* status, uint32_t code) {
+    return mbar_wait_spin(bar, parity, abort_flag, status, code);
+}
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
                                           uint32_t* status, uint32_t code) {
     if (mbar_try_wait(bar, parity)) return true;
     return mbar_wait_slow(bar, parity, abort_flag, status, code);
+}
+// the same wait with nothing called out of line: for kernels whose warps change their register
+// allowance (setmaxnreg), where a separately compiled callee would not know the caller's limit
+__device__ __forceinline__ bool mbar_wait_inl(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                              uint32_t* status, uint32_t code) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_spin(bar, parity, abort_flag, status, code);
+}
+// register re-allocation between the warpgroups of a CTA (every warp of the warpgroup executes it)
+template <int N> __device__ __forceinline__ void reg_dealloc() {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+}
+template <int N> __device__ __forceinline__ void reg_alloc() {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
@@ -105,6 +123,9 @@ template <int N> __device__ __forceinline__ void tma_store_wait_read() {
 }
 template <int N> __device__ __forceinline__ void tma_store_wait_all() {
     asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
