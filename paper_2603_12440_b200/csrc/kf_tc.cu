@@ -282,7 +282,12 @@ kf_status launch_tc_linear(const void* X, long long ldx, const void* W, long lon
     // the forms with row-norm and activation compiled in serve every CTA-pair call; the generic form
     // serves single row blocks and runs whenever a timing switch is set
     kf_status ls;
-    if (cta_group == 2 && p.debug == 0) {
+#ifdef KF_TC_COUNTERS                                   // build option: cycle counters in the specialised forms too
+    const bool spec = cta_group == 2 && (p.debug & ~1024) == 0;
+#else
+    const bool spec = cta_group == 2 && p.debug == 0;
+#endif
+    if (spec) {
         const TcLaunchArgs la = {grid, st, &tmX, &tmW, &tmY, &p};
         switch (rn.norm) {
         case KF_NORM_NONE: ls = tc_launch_spec_none(ep.act, la); break;

@@ -110,10 +110,50 @@ struct TcParams {
     long long timeout_cycles;   // limit of every bounded wait
 };
 
-// element-wise epilogue on 32 consecutive columns of one row, fast-math forms (bf16 output).
+// The epilogue arithmetic runs on pairs of adjacent columns with the packed fp32 instructions of
+// sm_100 (add / mul / fma on two floats at once): half the issue slots of the scalar forms.
+__device__ __forceinline__ float2 f2(float x, float y) { return make_float2(x, y); }
+__device__ __forceinline__ float2 f2(float x) { return make_float2(x, x); }
+
+// fast-math activation of a column pair (same forms as apply_act<false>, one special-function op per value)
+__device__ __forceinline__ float2 act_pair(const int act, const float2 z) {
+    switch (act) {
+    case KF_ACT_GELU_ERF: {
+        float2 z2 = __fmul2_rn(z, z);
+        z2.x = fminf(z2.x, 49.0f);
+        z2.y = fminf(z2.y, 49.0f);
+        float2 q = __ffma2_rn(f2(-0.0003514050040394068f), z2, f2(0.037005018442869186f));
+        q = __ffma2_rn(q, z2, f2(0.7975085377693176f));
+        const float2 u = __fmul2_rn(q, z);
+        const float2 hz = __fmul2_rn(z, f2(0.5f));
+        return __ffma2_rn(hz, f2(fast_tanh(u.x), fast_tanh(u.y)), hz);
+    }
+    case KF_ACT_GELU_TANH: {
+        const float2 z2 = __fmul2_rn(z, z);
+        const float2 q = __ffma2_rn(f2(0.7978845608028654f * 0.044715f), z2, f2(0.7978845608028654f));
+        const float2 u = __fmul2_rn(q, z);
+        const float2 hz = __fmul2_rn(z, f2(0.5f));
+        return __ffma2_rn(hz, f2(fast_tanh(u.x), fast_tanh(u.y)), hz);
+    }
+    case KF_ACT_SILU: {
+        const float2 hz = __fmul2_rn(z, f2(0.5f));
+        return __ffma2_rn(hz, f2(fast_tanh(hz.x), fast_tanh(hz.y)), hz);
+    }
+    case KF_ACT_RELU:
+        return f2(fmaxf(z.x, 0.0f), fmaxf(z.y, 0.0f));
+    case KF_ACT_SIGMOID: {
+        const float2 hz = __fmul2_rn(z, f2(0.5f));
+        return __ffma2_rn(f2(0.5f), f2(fast_tanh(hz.x), fast_tanh(hz.y)), f2(0.5f));
+    }
+    default:
+        return z;
+    }
+}
+
+// element-wise epilogue on 32 consecutive columns of one row (16 column pairs), bf16 output.
 // bias32: the 32 bias values as fp32 in shared memory (or nullptr); col0 = global column of a[0];
 // 8-column vectors at or beyond N are not read from the residual.
-__device__ __forceinline__ void epilogue32(float (&a)[32], const TcParams& p, const int act, const int debug,
+__device__ __forceinline__ void epilogue32(float2 (&a)[16], const TcParams& p, const int act, const int debug,
                                            const float* bias32, long long row, int col0, bool row_ok) {
     // the residual comes from global memory (often DRAM): issue its loads first, use them last
     const bool has_res = p.residual && row_ok && !(debug & 64);
@@ -129,44 +169,26 @@ __device__ __forceinline__ void epilogue32(float (&a)[32], const TcParams& p, co
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
             const float4 b = bp[q];
-            a[q * 4 + 0] += b.x; a[q * 4 + 1] += b.y; a[q * 4 + 2] += b.z; a[q * 4 + 3] += b.w;
+            a[2 * q] = __fadd2_rn(a[2 * q], f2(b.x, b.y));
+            a[2 * q + 1] = __fadd2_rn(a[2 * q + 1], f2(b.z, b.w));
         }
     }
     if (act != KF_ACT_NONE && !(debug & 32)) {
-        switch (act) {
-        case KF_ACT_GELU_ERF:
 #pragma unroll
-            for (int e = 0; e < 32; ++e) a[e] = apply_act<false>(KF_ACT_GELU_ERF, a[e]);
-            break;
-        case KF_ACT_GELU_TANH:
-#pragma unroll
-            for (int e = 0; e < 32; ++e) a[e] = apply_act<false>(KF_ACT_GELU_TANH, a[e]);
-            break;
-        case KF_ACT_SILU:
-#pragma unroll
-            for (int e = 0; e < 32; ++e) a[e] = apply_act<false>(KF_ACT_SILU, a[e]);
-            break;
-        case KF_ACT_RELU:
-#pragma unroll
-            for (int e = 0; e < 32; ++e) a[e] = fmaxf(a[e], 0.f);
-            break;
-        default:
-#pragma unroll
-            for (int e = 0; e < 32; ++e) a[e] = apply_act<false>(KF_ACT_SIGMOID, a[e]);
-            break;
-        }
+        for (int i = 0; i < 16; ++i) a[i] = act_pair(act, a[i]);
     }
     if (p.scale != 1.0f) {
+        const float2 sc = f2(p.scale);
 #pragma unroll
-        for (int e = 0; e < 32; ++e) a[e] *= p.scale;
+        for (int i = 0; i < 16; ++i) a[i] = __fmul2_rn(a[i], sc);
     }
     if (has_res) {
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-            float r[8];
-            unpack<__nv_bfloat16>(rv[q], r);
+            const uint32_t w[4] = {rv[q].x, rv[q].y, rv[q].z, rv[q].w};
 #pragma unroll
-            for (int e = 0; e < 8; ++e) a[q * 8 + e] += r[e];
+            for (int j = 0; j < 4; ++j)     // a bf16 pair widens to fp32 by shifting / masking the word
+                a[q * 4 + j] = __fadd2_rn(a[q * 4 + j], f2(__uint_as_float(w[j] << 16), __uint_as_float(w[j] & 0xFFFF0000u)));
         }
     }
 }
@@ -193,7 +215,14 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     const int debug = kGeneric ? p.debug : 0;
     // cycle counters of the generic form (debug bit 1024): how long the MMA thread waits for operands
     // and for a free accumulator, how long the epilogue waits, holds the accumulator and works
-    auto tick = [&]() -> long long { return kGeneric ? clock64() : 0ll; };
+#ifdef KF_TC_COUNTERS                                   // build option: the specialised forms count too
+    constexpr bool kCount = true;
+    const bool count_on = (p.debug & 1024) != 0;
+#else
+    constexpr bool kCount = kGeneric;
+    const bool count_on = (debug & 1024) != 0;
+#endif
+    auto tick = [&]() -> long long { return kCount ? clock64() : 0ll; };
     using C = Cfg<CG>;
     constexpr int kStages = C::kStages;
     constexpr uint32_t kSmemB = C::kSmemB, kBBytes = C::kBBytes;
@@ -332,7 +361,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
                 }
                 if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
             }
-            if (debug & 1024) {
+            if (count_on) {
                 unsigned long long* t64 = reinterpret_cast<unsigned long long*>(p.status);
                 atomicAdd(t64 + 6, (unsigned long long)tw_acc);
                 atomicAdd(t64 + 7, (unsigned long long)tw_full);
@@ -394,45 +423,66 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             }
             te_s1 += tick() - te1;
 
-            // element-wise epilogue in place, per-row statistics of the sub-tile (4 independent accumulators each)
+            // element-wise epilogue in place on column pairs, per-row statistics of the sub-tile; columns
+            // beyond N (ragged last chunk) are set to the neutral value of the statistic
             float st_shift = 0.f, st_s1 = 0.f, st_s2 = 0.f, st_scale = 1.f, mult = 1.f;
-            float s1[4] = {0.f, 0.f, 0.f, 0.f}, s2[4] = {0.f, 0.f, 0.f, 0.f};
+            float2 s1[2] = {f2(0.f), f2(0.f)}, s2[2] = {f2(0.f), f2(0.f)};
             float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY}, am[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int c = 0; c < kSub / 32; ++c) {
                 if (c < nchunks) {
-                    float a[32];
+                    float2 a[16];
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) a[e] = __uint_as_float(v[c][e]);
+                    for (int i = 0; i < 16; ++i) a[i] = f2(__uint_as_float(v[c][2 * i]), __uint_as_float(v[c][2 * i + 1]));
                     epilogue32(a, p, act, debug, bias_t ? bias_t + c * 32 : nullptr, row, n0 + cb + c * 32, row_ok);
                     const bool full = (c + 1) * 32 <= ncols;
                     if (norm == KF_NORM_SOFTMAX) {
+                        if (!full) {
 #pragma unroll
-                        for (int e = 0; e < 32; ++e)
-                            if (full || c * 32 + e < ncols) mx[e & 3] = fmaxf(mx[e & 3], a[e]);
-                    } else if (norm != KF_NORM_NONE) {
-                        if (norm == KF_NORM_LAYERNORM) {
-                            if (c == 0) st_shift = a[0];
-#pragma unroll
-                            for (int e = 0; e < 32; ++e) a[e] -= st_shift;
+                            for (int i = 0; i < 16; ++i) {
+                                if (c * 32 + 2 * i >= ncols) a[i].x = -INFINITY;
+                                if (c * 32 + 2 * i + 1 >= ncols) a[i].y = -INFINITY;
+                            }
                         }
 #pragma unroll
-                        for (int e = 0; e < 32; ++e)
-                            if (full || c * 32 + e < ncols) {
-                                s1[e & 3] += a[e];
-                                s2[e & 3] = fmaf(a[e], a[e], s2[e & 3]);
-                                am[e & 3] = fmaxf(am[e & 3], fabsf(a[e]));
+                        for (int i = 0; i < 16; ++i) {
+                            mx[(2 * i) & 3] = fmaxf(mx[(2 * i) & 3], a[i].x);
+                            mx[(2 * i + 1) & 3] = fmaxf(mx[(2 * i + 1) & 3], a[i].y);
+                        }
+                    } else if (norm != KF_NORM_NONE) {
+                        if (norm == KF_NORM_LAYERNORM) {
+                            if (c == 0) st_shift = a[0].x;
+                            const float2 ns = f2(-st_shift);
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) a[i] = __fadd2_rn(a[i], ns);
+                        }
+                        if (!full) {
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) {
+                                if (c * 32 + 2 * i >= ncols) a[i].x = 0.f;
+                                if (c * 32 + 2 * i + 1 >= ncols) a[i].y = 0.f;
                             }
+                        }
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            s1[i & 1] = __fadd2_rn(s1[i & 1], a[i]);
+                            s2[i & 1] = __ffma2_rn(a[i], a[i], s2[i & 1]);
+                            am[(2 * i) & 3] = fmaxf(am[(2 * i) & 3], fabsf(a[i].x));
+                            am[(2 * i + 1) & 3] = fmaxf(am[(2 * i + 1) & 3], fabsf(a[i].y));
+                        }
                     }
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) v[c][e] = __float_as_uint(a[e]);
+                    for (int i = 0; i < 16; ++i) {
+                        v[c][2 * i] = __float_as_uint(a[i].x);
+                        v[c][2 * i + 1] = __float_as_uint(a[i].y);
+                    }
                 }
             }
             if (norm == KF_NORM_SOFTMAX) {
                 st_shift = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
             } else if (norm != KF_NORM_NONE) {
-                st_s1 = (s1[0] + s1[1]) + (s1[2] + s1[3]);
-                st_s2 = (s2[0] + s2[1]) + (s2[2] + s2[3]);
+                st_s1 = (s1[0].x + s1[0].y) + (s1[1].x + s1[1].y);
+                st_s2 = (s2[0].x + s2[0].y) + (s2[1].x + s2[1].y);
                 const float amax = fmaxf(fmaxf(am[0], am[1]), fmaxf(am[2], am[3]));
                 // power-of-two block scale: stored fp16 values lie in (-2, 2)
                 uint32_t eb = (__float_as_uint(amax) >> 23) & 0xFFu;
@@ -442,30 +492,31 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             }
             // 16-bit pack and store: the result (no row-norm) or the intermediate the finishing kernel rescales
             {
-                float l4[4] = {0.f, 0.f, 0.f, 0.f};
-                const float ms = st_shift * kLog2e;
+                float2 l2[2] = {f2(0.f), f2(0.f)};
+                const float2 nms = f2(-st_shift * kLog2e), l2e = f2(kLog2e), m2 = f2(mult);
 #pragma unroll
                 for (int c = 0; c < kSub / 32; ++c) {
                     if (c < nchunks) {
-                        float a[32];
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) a[e] = __uint_as_float(v[c][e]);
                         uint32_t w[16];
                         if (norm == KF_NORM_NONE) {
 #pragma unroll
-                            for (int e = 0; e < 16; ++e) w[e] = pack_bf16(a[2 * e], a[2 * e + 1]);
+                            for (int i = 0; i < 16; ++i)
+                                w[i] = pack_bf16(__uint_as_float(v[c][2 * i]), __uint_as_float(v[c][2 * i + 1]));
                         } else if (norm == KF_NORM_SOFTMAX) {
-                            const bool full = (c + 1) * 32 <= ncols;
 #pragma unroll
-                            for (int e = 0; e < 32; ++e) {
-                                a[e] = fast_ex2(fmaf(a[e], kLog2e, -ms));
-                                if (full || c * 32 + e < ncols) l4[e & 3] += a[e];
+                            for (int i = 0; i < 16; ++i) {      // columns beyond N hold -inf: exp gives 0
+                                const float2 t = __ffma2_rn(f2(__uint_as_float(v[c][2 * i]), __uint_as_float(v[c][2 * i + 1])),
+                                                            l2e, nms);
+                                const float2 ex = f2(fast_ex2(t.x), fast_ex2(t.y));
+                                l2[i & 1] = __fadd2_rn(l2[i & 1], ex);
+                                w[i] = pack_bf16(ex.x, ex.y);
                             }
-#pragma unroll
-                            for (int e = 0; e < 16; ++e) w[e] = pack_bf16(a[2 * e], a[2 * e + 1]);
                         } else {
 #pragma unroll
-                            for (int e = 0; e < 16; ++e) w[e] = pack_f16(a[2 * e] * mult, a[2 * e + 1] * mult);
+                            for (int i = 0; i < 16; ++i) {
+                                const float2 t = __fmul2_rn(f2(__uint_as_float(v[c][2 * i]), __uint_as_float(v[c][2 * i + 1])), m2);
+                                w[i] = pack_f16(t.x, t.y);
+                            }
                         }
                         if (debug & 128) {
                             if (row_ok && !(debug & 8))
@@ -495,7 +546,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
                         }
                     }
                 }
-                if (norm == KF_NORM_SOFTMAX) st_s1 = (l4[0] + l4[1]) + (l4[2] + l4[3]);
+                if (norm == KF_NORM_SOFTMAX) st_s1 = (l2[0].x + l2[0].y) + (l2[1].x + l2[1].y);
             }
             if (debug & 256) {                            // timing experiment: a 5 us longer epilogue
                 const long long t0 = clock64();
@@ -508,7 +559,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             te_work += tick() - te1;
         }
         if (lane == 0) tma_store_wait_all<0>();              // the staging buffers are read, Y is written
-        if ((debug & 1024) && warp == kRoleWarps && lane == 0) {
+        if (count_on && warp == kRoleWarps && lane == 0) {
             unsigned long long* t64 = reinterpret_cast<unsigned long long*>(p.status);
             atomicAdd(t64 + 4, (unsigned long long)te_wait);
             atomicAdd(t64 + 5, (unsigned long long)te_work);
