@@ -147,6 +147,19 @@ def test_tc_rownorm_split_n(kf, norm, M, N, K):
     assert_parity(run(kf, p), oracle_of(p), "bf16", f"{norm} {M}x{N}x{K}")
 
 
+@pytest.mark.parametrize("norm", ["none", "softmax", "layernorm", "rmsnorm"])
+@pytest.mark.parametrize("act", ACTS)
+def test_tc_every_specialised_kernel(kf, act, norm):
+    """CTA-pair calls run a kernel compiled for their (row-norm, activation) pair: each of the 24
+    instantiations against the oracle on a ragged 3 x 4-tile problem, with and without a residual."""
+    i = ACTS.index(act)
+    p = make("bf16", 290, 776, 136, seed=300 + 4 * i, act=act, norm=norm, bias=i % 3 != 0, res=i % 2 == 0,
+             scale=[1.0, 0.5, 2.0][i % 3])
+    cfg = kf.tile_config(p.M, p.N, p.K, torch.bfloat16, norm)
+    assert cfg["kernel"] == 3 and cfg["cta_group"] == 2
+    assert_parity(run(kf, p), oracle_of(p), "bf16", f"{act} {norm}")
+
+
 def test_tc_layernorm_with_mean_far_from_zero(kf):
     # sigmoid outputs sit near 0.5 with a small spread: the per-tile shift keeps the deviations exact
     p = make("bf16", 200, 1536, 256, seed=27, act="sigmoid", norm="layernorm", res=False, std=0.01)
