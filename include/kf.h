@@ -144,8 +144,14 @@ kf_status kf_row_rmsnorm(const void *X, int64_t ldx, const void *gamma, float ep
  * ep and rn are HOST pointers (pinned memory makes the copies asynchronous), tightly packed
  * (pitch = row length).  `dev` is caller-owned device memory of at least
  * kf_host_call_bytes(M,N,K,dt,has_residual,norm) bytes, 256-byte aligned; the call copies the
- * inputs into it on `stream`, runs the device path there and copies Y back to the host.  The
- * result is complete when `stream` has been synchronised by the caller.
+ * inputs into it, runs the device path there and copies Y back to the host.  The result is
+ * complete when `stream` has been synchronised by the caller.  Small calls run entirely on
+ * `stream`.  Large bf16 calls (at least 1024 rows and 4 Mi outputs) are cut into up to 8 chunks of
+ * rows -- rows are independent -- whose input copy, computation and output copy run on three
+ * internal streams of the device (created on first use), so that the copy of one chunk's result
+ * overlaps the next chunk's work; that work is ordered after everything already in `stream`, and
+ * `stream` waits for all of it before the call returns control of the stream to the caller.  The
+ * bytes written to Y are those of one device call on the whole problem either way.
  */
 kf_status kf_linear_epilogue_rownorm_host(const void *X, const void *W, void *Y, int64_t M,
                                           int64_t N, int64_t K, kf_dtype dt,

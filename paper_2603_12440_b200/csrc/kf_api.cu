@@ -3,6 +3,7 @@
 // except in kf_check_device_status.
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 
 #include "kf_tc.cuh"
 
@@ -234,6 +235,53 @@ size_t kf_host_call_bytes(int64_t M, int64_t N, int64_t K, kf_dtype dt, int has_
     return b;
 }
 
+// ---- host-buffer call, pipelined over row chunks ------------------------------------------------
+// Rows are independent, so a large call is cut into chunks of rows: while chunk c is computed, the
+// inputs of chunk c+1 come in and the result of chunk c-1 goes out, each on its own internal
+// stream (PCIe carries both directions at once).  Everything is ordered after the work already in
+// `stream`, and `stream` waits for all of it at the end.
+namespace {
+
+constexpr int kMaxChunks = 8;
+
+struct HostPipe {
+    cudaStream_t in = nullptr, cmp = nullptr, out = nullptr;
+    cudaEvent_t start = nullptr, weights = nullptr, rows_in[kMaxChunks] = {}, computed[kMaxChunks] = {};
+    cudaEvent_t end_in = nullptr, end_cmp = nullptr, end_out = nullptr;
+    bool ok = false;
+};
+
+std::mutex g_pipe_mu;
+
+HostPipe* host_pipe() {                                  // per device, created on first use; g_pipe_mu held
+    static HostPipe pipes[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    HostPipe& p = pipes[dev];
+    if (!p.ok) {
+        bool good = cudaStreamCreateWithFlags(&p.in, cudaStreamNonBlocking) == cudaSuccess &&
+                    cudaStreamCreateWithFlags(&p.cmp, cudaStreamNonBlocking) == cudaSuccess &&
+                    cudaStreamCreateWithFlags(&p.out, cudaStreamNonBlocking) == cudaSuccess;
+        auto ev = [&](cudaEvent_t* e) { good = good && cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess; };
+        ev(&p.start); ev(&p.weights); ev(&p.end_in); ev(&p.end_cmp); ev(&p.end_out);
+        for (int c = 0; c < kMaxChunks; ++c) { ev(&p.rows_in[c]); ev(&p.computed[c]); }
+        if (!good) return nullptr;
+        p.ok = true;
+    }
+    return &p;
+}
+
+// rows per chunk (a multiple of 256 = one CTA-pair row unit), or 0 when the call is not worth cutting
+int64_t host_chunk_rows(int64_t M, int64_t N, int64_t K, int dt) {
+    if (dt != KF_BF16 || K <= 0 || M < 1024 || (size_t)M * N < ((size_t)4 << 20)) return 0;
+    int64_t chunks = M / 512;
+    if (chunks > kMaxChunks) chunks = kMaxChunks;
+    const int64_t rows = ((M + chunks - 1) / chunks + 255) / 256 * 256;
+    return rows < M ? rows : 0;
+}
+
+}  // namespace
+
 kf_status kf_linear_epilogue_rownorm_host(const void* X, const void* W, void* Y, int64_t M, int64_t N, int64_t K,
                                           kf_dtype dt, const kf_epilogue* ep, const kf_rownorm* rn, void* dev,
                                           size_t dev_bytes, void* stream) {
@@ -256,6 +304,69 @@ kf_status kf_linear_epilogue_rownorm_host(const void* X, const void* W, void* Y,
         if (host && bytes) copy_ok &= cudaMemcpyAsync(d, host, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
         return host ? d : nullptr;
     };
+    const int64_t chunk_rows = host_chunk_rows(M, N, K, (int)dt);
+    if (chunk_rows > 0) {
+        std::lock_guard<std::mutex> lock(g_pipe_mu);        // the internal streams and events are shared per device
+        HostPipe* hp = host_pipe();
+        if (!hp) return KF_ERR_CUDA;
+        bool good = true;
+        auto chk = [&](cudaError_t e) { good = good && e == cudaSuccess; };
+        auto put = [&](const void* host, size_t bytes) -> uint8_t* {      // reserve, and copy on the input stream
+            uint8_t* d = cur;
+            cur += round256(bytes);
+            if (host && bytes) chk(cudaMemcpyAsync(d, host, bytes, cudaMemcpyHostToDevice, hp->in));
+            return host ? d : nullptr;
+        };
+        chk(cudaEventRecord(hp->start, st));
+        chk(cudaStreamWaitEvent(hp->in, hp->start, 0));
+        chk(cudaStreamWaitEvent(hp->cmp, hp->start, 0));
+        chk(cudaStreamWaitEvent(hp->out, hp->start, 0));
+        uint8_t* dXc = cur; cur += round256((size_t)M * K * es);         // rows of X arrive chunk by chunk below
+        uint8_t* dWc = put(W, (size_t)N * K * es);
+        uint8_t* dYc = cur; cur += round256((size_t)M * N * es);
+        uint8_t* dRc = nullptr;
+        if (has_res) { dRc = cur; cur += round256((size_t)M * N * es); }
+        kf_epilogue dep{nullptr, KF_ACT_NONE, 1.0f, nullptr, 0};
+        if (ep) dep = *ep;
+        dep.bias = put(ep ? ep->bias : nullptr, (size_t)N * es);
+        kf_rownorm drn{KF_NORM_NONE, nullptr, nullptr, 0.f};
+        if (rn) drn = *rn;
+        drn.gamma = put(rn ? rn->gamma : nullptr, (size_t)N * es);
+        drn.beta = put(rn ? rn->beta : nullptr, (size_t)N * es);
+        void* ws = cur;
+        const size_t ws_bytes = kf_workspace_bytes(M, N, K, dt, (kf_norm)norm);
+        chk(cudaMemsetAsync(ws, 0, kStatusBytes, hp->cmp));
+        chk(cudaEventRecord(hp->weights, hp->in));
+        chk(cudaStreamWaitEvent(hp->cmp, hp->weights, 0));
+        if (!good) return KF_ERR_CUDA;
+        int c = 0;
+        for (int64_t r0 = 0; r0 < M; r0 += chunk_rows, ++c) {
+            const int64_t rows = r0 + chunk_rows <= M ? chunk_rows : M - r0;
+            chk(cudaMemcpyAsync(dXc + (size_t)r0 * K * es, static_cast<const uint8_t*>(X) + (size_t)r0 * K * es,
+                                (size_t)rows * K * es, cudaMemcpyHostToDevice, hp->in));
+            if (has_res)
+                chk(cudaMemcpyAsync(dRc + (size_t)r0 * N * es, static_cast<const uint8_t*>(ep->residual) + (size_t)r0 * N * es,
+                                    (size_t)rows * N * es, cudaMemcpyHostToDevice, hp->in));
+            chk(cudaEventRecord(hp->rows_in[c], hp->in));
+            chk(cudaStreamWaitEvent(hp->cmp, hp->rows_in[c], 0));
+            if (!good) return KF_ERR_CUDA;
+            if (has_res) { dep.residual = dRc + (size_t)r0 * N * es; dep.ldr = N; }
+            s = linear_impl(dXc + (size_t)r0 * K * es, K, dWc, K, dYc + (size_t)r0 * N * es, N, rows, N, K, (int)dt, &dep, &drn,
+                            ws, ws_bytes, hp->cmp);
+            if (s != KF_OK) return s;
+            chk(cudaEventRecord(hp->computed[c], hp->cmp));
+            chk(cudaStreamWaitEvent(hp->out, hp->computed[c], 0));
+            chk(cudaMemcpyAsync(static_cast<uint8_t*>(Y) + (size_t)r0 * N * es, dYc + (size_t)r0 * N * es, (size_t)rows * N * es,
+                                cudaMemcpyDeviceToHost, hp->out));
+        }
+        chk(cudaEventRecord(hp->end_in, hp->in));
+        chk(cudaEventRecord(hp->end_cmp, hp->cmp));
+        chk(cudaEventRecord(hp->end_out, hp->out));
+        chk(cudaStreamWaitEvent(st, hp->end_in, 0));
+        chk(cudaStreamWaitEvent(st, hp->end_cmp, 0));
+        chk(cudaStreamWaitEvent(st, hp->end_out, 0));
+        return good ? KF_OK : KF_ERR_CUDA;
+    }
     void* dX = stage(K > 0 ? X : nullptr, (size_t)M * K * es);
     void* dW = stage(K > 0 ? W : nullptr, (size_t)N * K * es);
     void* dY = cur;

@@ -217,18 +217,26 @@ def test_tc_deterministic_and_fresh_each_call(kf):
     assert not torch.equal(y1, y3)
 
 
-def test_host_buffer_call_matches_device_call(kf):
-    p = make("bf16", 300, 520, 200, seed=33, act="gelu_erf", norm="layernorm", res=True)
+@pytest.mark.parametrize("M,N,K,norm,res", [(300, 520, 200, "layernorm", True),      # one piece
+                                             (1300, 4104, 136, "layernorm", True),     # two row chunks, ragged
+                                             (2100, 2056, 72, "softmax", False),       # four row chunks
+                                             (1536, 4096, 64, "none", True)])
+def test_host_buffer_call_matches_device_call(kf, M, N, K, norm, res):
+    """The host-buffer form cuts large calls into row chunks that it copies in, computes and copies out on
+    internal streams; the bytes it returns are those of the device call on the whole problem."""
+    p = make("bf16", M, N, K, seed=33 + M, act="gelu_erf", norm=norm, res=res)
     d = problem_to_device(p)
     ydev = kf.linear_epilogue_rownorm(d["X"], d["W"], d["bias"], p.act, p.scale, d["residual"], p.norm,
                                       d["gamma"], d["beta"], p.eps)
     h = {k: (v.cpu().pin_memory() if v is not None else None) for k, v in d.items()}
-    out = torch.empty(p.M, p.N, dtype=torch.bfloat16).pin_memory()
-    arena = torch.empty(kf.host_call_bytes(p.M, p.N, p.K, torch.bfloat16, True, p.norm), dtype=torch.uint8, device="cuda")
-    kf.linear_epilogue_rownorm_host(h["X"], h["W"], out, arena, h["bias"], p.act, p.scale, h["residual"], p.norm,
-                                    h["gamma"], h["beta"], p.eps)
-    torch.cuda.synchronize()
-    assert torch.equal(out, ydev.cpu())
+    arena = torch.empty(kf.host_call_bytes(p.M, p.N, p.K, torch.bfloat16, res, p.norm), dtype=torch.uint8, device="cuda")
+    for _ in range(2):                                  # twice: the internal streams and events are reused
+        out = torch.full((p.M, p.N), float("nan"), dtype=torch.bfloat16).pin_memory()
+        kf.linear_epilogue_rownorm_host(h["X"], h["W"], out, arena, h["bias"], p.act, p.scale, h["residual"], p.norm,
+                                        h["gamma"], h["beta"], p.eps)
+        torch.cuda.synchronize()
+        assert torch.equal(out, ydev.cpu())
+    assert_parity(to_f64(ydev), oracle_of(p), "bf16", f"host {M}x{N}x{K} {norm}")
 
 
 def test_degenerate_sizes(kf):
