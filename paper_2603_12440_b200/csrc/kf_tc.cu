@@ -17,6 +17,7 @@ namespace kf {
 namespace {
 
 constexpr int kFinWarps = 8;
+constexpr int kFinBatch = 4;                            // 16-byte vectors per lane and batch in the finishing kernel
 
 template <bool IS_MAX>
 __device__ __forceinline__ float fin_group_reduce(float v, int wpr, int warp, float* red) {
@@ -32,7 +33,7 @@ __device__ __forceinline__ float fin_group_reduce(float v, int wpr, int warp, fl
 }
 
 __global__ void __launch_bounds__(kFinWarps * 32)
-tc_rownorm_finish_kernel(__nv_bfloat16* Y, long long ldy, int M, int N, int nsub, int wpr,
+tc_rownorm_finish_kernel(__nv_bfloat16* Y, long long ldy, int M, int N, int nsub, int wpr, int staged,
                          const float4* __restrict__ partials, int norm, const __nv_bfloat16* __restrict__ gamma,
                          const __nv_bfloat16* __restrict__ beta, float eps) {
     extern __shared__ float2 coef_smem[];               // per row of the CTA: nsub x {multiplier, offset}
@@ -95,7 +96,66 @@ tc_rownorm_finish_kernel(__nv_bfloat16* Y, long long ldy, int M, int N, int nsub
     const uint4* gv = reinterpret_cast<const uint4*>(gamma);
     const uint4* bv = reinterpret_cast<const uint4*>(beta);
     const int NV = N / 8;
-    constexpr int U = 4;                                 // vectors in flight per lane
+    constexpr int U = kFinBatch;                         // vectors per lane and batch
+    // one 16-byte piece of the intermediate -> normalised bf16
+    auto piece = [&](uint4 raw, int idx) -> uint4 {
+        float f[8];
+        const float2 c = coef[idx / (kSub / 8)];
+        if (norm == KF_NORM_SOFTMAX) {
+            unpack<__nv_bfloat16>(raw, f);
+            const float k = c.x * rstd;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) f[e] *= k;
+        } else {
+            unpack_f16x8(raw, f);
+            float g[8], b[8];
+            if (gamma) unpack<__nv_bfloat16>(__ldg(gv + idx), g);
+            if (beta && norm == KF_NORM_LAYERNORM) unpack<__nv_bfloat16>(__ldg(bv + idx), b);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                float o = fmaf(f[e], c.x, c.y) * rstd;
+                if (gamma) o *= g[e];
+                if (beta && norm == KF_NORM_LAYERNORM) o += b[e];
+                f[e] = o;
+            }
+        }
+        return pack<__nv_bfloat16>(f);
+    };
+    if (staged) {
+        // one warp per row: the row streams through two warp-private 2 KiB buffers filled by cp.async, so
+        // that the loads of the next batch are in flight while this one is rescaled and stored (every
+        // lane reads back only the pieces it requested itself: no barrier, no bank conflict)
+        const uint32_t sbuf = smem_u32(coef_smem + (size_t)rows_per_cta * nsub) + (uint32_t)warp * (2u * U * 32u * 16u);
+        auto request = [&](int b, int i0) {
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int idx = i0 + u * 32;
+                if (idx < NV)
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sbuf + (uint32_t)((b * U + u) * 32 + lane) * 16u),
+                                 "l"(yr + idx)
+                                 : "memory");
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        };
+        int b = 0;
+        request(0, lane);
+        for (int i0 = lane; i0 < NV; i0 += 32 * U, b ^= 1) {
+            request(b ^ 1, i0 + 32 * U);                 // (an empty group past the end of the row)
+            asm volatile("cp.async.wait_group 1;" ::: "memory");
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int idx = i0 + u * 32;
+                if (idx >= NV) break;
+                uint4 raw;
+                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                             : "=r"(raw.x), "=r"(raw.y), "=r"(raw.z), "=r"(raw.w)
+                             : "r"(sbuf + (uint32_t)((b * U + u) * 32 + lane) * 16u)
+                             : "memory");
+                yr[idx] = piece(raw, idx);
+            }
+        }
+        return;
+    }
     for (int i0 = gt; i0 < NV; i0 += gsize * U) {
         uint4 raw[U];
 #pragma unroll
@@ -107,27 +167,7 @@ tc_rownorm_finish_kernel(__nv_bfloat16* Y, long long ldy, int M, int N, int nsub
         for (int u = 0; u < U; ++u) {
             const int idx = i0 + u * gsize;
             if (idx >= NV) break;
-            float f[8];
-            const float2 c = coef[idx / (kSub / 8)];
-            if (norm == KF_NORM_SOFTMAX) {
-                unpack<__nv_bfloat16>(raw[u], f);
-                const float k = c.x * rstd;
-#pragma unroll
-                for (int e = 0; e < 8; ++e) f[e] *= k;
-            } else {
-                unpack_f16x8(raw[u], f);
-                float g[8], b[8];
-                if (gamma) unpack<__nv_bfloat16>(__ldg(gv + idx), g);
-                if (beta && norm == KF_NORM_LAYERNORM) unpack<__nv_bfloat16>(__ldg(bv + idx), b);
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    float o = fmaf(f[e], c.x, c.y) * rstd;
-                    if (gamma) o *= g[e];
-                    if (beta && norm == KF_NORM_LAYERNORM) o += b[e];
-                    f[e] = o;
-                }
-            }
-            yr[idx] = pack<__nv_bfloat16>(f);
+            yr[idx] = piece(raw[u], idx);
         }
     }
 }
@@ -277,8 +317,25 @@ kf_status launch_tc_linear(const void* X, long long ldx, const void* W, long lon
     }();
     if (env_wpr == 1 || env_wpr == 2 || env_wpr == 4 || env_wpr == 8) wpr = env_wpr;
     const int fin_rows = kFinWarps / wpr;
-    const size_t fin_smem = (size_t)p.nsub * fin_rows * sizeof(float2);
-    if (rn.norm != KF_NORM_NONE && fin_smem > 48 * 1024) return KF_ERR_UNSUPPORTED;   // N beyond ~780k
+    const size_t fin_coef = (size_t)p.nsub * fin_rows * sizeof(float2);
+    if (rn.norm != KF_NORM_NONE && fin_coef > 48 * 1024) return KF_ERR_UNSUPPORTED;   // N beyond ~780k
+    // one warp per row: the rows stream through cp.async staging buffers behind the coefficient table
+    static const bool env_nostage = std::getenv("KF_FIN_NOSTAGE") != nullptr;
+    const int fin_staged = (wpr == 1 && !env_nostage) ? 1 : 0;
+    const size_t fin_smem = fin_coef + (fin_staged ? (size_t)kFinWarps * 2 * kFinBatch * 32 * 16 : 0);
+    if (rn.norm != KF_NORM_NONE && fin_staged) {
+        static std::mutex mu;
+        static bool done[64] = {};
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return KF_ERR_CUDA;
+        std::lock_guard<std::mutex> lock(mu);
+        if (!done[dev]) {
+            if (cudaFuncSetAttribute(tc_rownorm_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024) !=
+                cudaSuccess)
+                return KF_ERR_CUDA;
+            done[dev] = true;
+        }
+    }
     // the forms with row-norm and activation compiled in serve every CTA-pair call; the generic form
     // serves single row blocks and runs whenever a timing switch is set
     kf_status ls;
@@ -307,7 +364,7 @@ kf_status launch_tc_linear(const void* X, long long ldx, const void* W, long lon
 
     if (rn.norm != KF_NORM_NONE) {
         tc_rownorm_finish_kernel<<<(unsigned)((M + fin_rows - 1) / fin_rows), kFinWarps * 32, fin_smem, st>>>(
-            static_cast<__nv_bfloat16*>(Y), ldy, (int)M, (int)N, p.nsub, wpr, p.partials, rn.norm,
+            static_cast<__nv_bfloat16*>(Y), ldy, (int)M, (int)N, p.nsub, wpr, fin_staged, p.partials, rn.norm,
             static_cast<const __nv_bfloat16*>(rn.gamma), static_cast<const __nv_bfloat16*>(rn.beta), rn.eps);
         if (cudaGetLastError() != cudaSuccess) return KF_ERR_CUDA;
     }
