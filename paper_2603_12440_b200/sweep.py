@@ -2,8 +2,8 @@
 
 The paper's templated-kernel step (Section 3.4) instantiates a kernel for every parameter setting,
 times each and keeps the fastest; this is that step for the choices this library exposes:
-CTAs per MMA and grid size of the tensor-core kernel, and threads per row / ring on-off of the row
-kernels.  Each candidate runs in a fresh process (the overrides are read once per process):
+CTAs per MMA and grid size of the tensor-core kernel, its generic against its specialised form, the
+variants of the finishing pass, and threads per row / ring on-off of the row kernels.  Each candidate runs in a fresh process (the overrides are read once per process):
 
     python -m paper_2603_12440_b200.sweep --config c3 [--steps 30]
 
@@ -31,10 +31,15 @@ def candidates(config: str):
         yield {}, "table default"
         yield {"KF_TILE_OVERRIDE": "kernel=2"}, "tiled CUDA-core kernel + row kernel"
         return
-    for cg in (1, 2):
+    for cg in (2, 1):               # cg=1 on more than one row block runs the generic form of the kernel
         for grid in (0, 144, 128, 112, 96):
             ov = f"cg={cg}" + (f",grid={grid}" if grid else "")
             yield {"KF_TILE_OVERRIDE": ov}, ov
+    yield {"KF_TC_DEBUG": "128"}, "cg=2, generic form of the kernel, register stores"
+    if config in ("c4", "c5"):      # finishing pass of the split-N row-norm
+        yield {"KF_FIN_NOSTAGE": "1"}, "cg=2, finishing pass without cp.async staging"
+        for wpr in (2, 4):
+            yield {"KF_FIN_WPR": str(wpr)}, f"cg=2, finishing pass with {wpr} warps per row"
 
 
 def main():
