@@ -160,6 +160,16 @@ def test_tc_every_specialised_kernel(kf, act, norm):
     assert_parity(run(kf, p), oracle_of(p), "bf16", f"{act} {norm}")
 
 
+@pytest.mark.parametrize("M,N,K,norm", [(20000, 264, 72, "layernorm"),       # tall: 157 row blocks
+                                         (130, 98312, 64, "softmax"),         # 769 sub-tiles per row: the finishing
+                                         (260, 90120, 40, "layernorm")])      # pass shares a row between two warps
+def test_tc_tall_and_very_wide_rownorm(kf, M, N, K, norm):
+    p = make("bf16", M, N, K, seed=61 + K, act="silu", norm=norm, res=False)
+    cfg = kf.tile_config(M, N, K, torch.bfloat16, norm)
+    assert cfg["kernel"] == 3 and cfg["row_scheme"] == 2
+    assert_parity(run(kf, p), oracle_of(p), "bf16", f"{norm} {M}x{N}x{K}")
+
+
 def test_tc_layernorm_with_mean_far_from_zero(kf):
     # sigmoid outputs sit near 0.5 with a small spread: the per-tile shift keeps the deviations exact
     p = make("bf16", 200, 1536, 256, seed=27, act="sigmoid", norm="layernorm", res=False, std=0.01)
