@@ -7,7 +7,9 @@ variants of the finishing pass, and threads per row / ring on-off of the row ker
 
     python -m paper_2603_12440_b200.sweep --config c3 [--steps 30]
 
-Needs a B200; prints one JSON line per candidate and the winner.
+Needs a B200; prints one JSON line per candidate, the winner, and the candidates filed in the archive
+of kernel variants (descriptor cells, fitness against the same operator in plain PyTorch, gradient
+estimates: the paper's Sections 3.2 and 3.3 without the language model).
 """
 from __future__ import annotations
 
@@ -42,6 +44,79 @@ def candidates(config: str):
             yield {"KF_FIN_WPR": str(wpr)}, f"cg=2, finishing pass with {wpr} warps per row"
 
 
+def descriptors(config: str, label: str):
+    """(d_mem, d_algo, d_sync) of a candidate on the paper's scales (Section 3.2, "Kernel-Specific
+    Behavioral Descriptors"): d_mem 1 coalesced / vectorised, 2 shared-memory tiling, 3 multi-level hierarchy
+    (TMA ring + TMEM / registers); d_algo 0 direct translation (separate kernels), 1 fused single pass,
+    2 reformulated (online normalisation over split rows); d_sync 1 work-group barriers, 2 sub-group
+    shuffles, 3 global coordination (partials in global memory + a second pass)."""
+    if config == "c2":
+        return (3, 1, 2) if label.startswith("ring") else (1, 1, 2)
+    if config == "c1":
+        return (2, 1, 1) if label.startswith("table") else (2, 0, 1)
+    if config == "c3":
+        return (3, 1, 1)
+    return (3, 2, 3)
+
+
+def torch_baseline_ms(config: str, steps: int):
+    """The same operator written as plain PyTorch calls (the baseline the paper's speed-ups and its
+    fitness function refer to), timed like the candidates: flushed L2, CUDA events, median."""
+    import torch
+    import torch.nn.functional as F
+    sys.path.insert(0, str(ROOT))
+    import bench
+    from paper_2603_12440_b200 import inputs
+    p = inputs.config(int(config[1]))
+    d = inputs.problem_to_torch(p)
+    act = {"none": lambda z: z, "gelu_erf": F.gelu, "gelu_tanh": lambda z: F.gelu(z, approximate="tanh"), "silu": F.silu,
+           "relu": F.relu, "sigmoid": torch.sigmoid}[p.act]
+
+    def call():
+        y = d["X"] if p.W is None else F.linear(d["X"], d["W"], d["bias"])
+        if p.W is not None:
+            y = act(y)
+            if p.scale != 1.0:
+                y = y * p.scale
+            if d["residual"] is not None:
+                y = y + d["residual"]
+        if p.norm == "softmax":
+            y = torch.softmax(y, dim=-1)
+        elif p.norm == "layernorm":
+            y = F.layer_norm(y, (p.N,), d["gamma"], d["beta"], p.eps)
+        elif p.norm == "rmsnorm":
+            y = F.rms_norm(y, (p.N,), d["gamma"], p.eps)
+        return y
+
+    buf = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    ms, _ = bench.time_steps(call, steps, 3, lambda: buf.fill_(1))
+    return bench.median(ms)
+
+
+def file_results(config: str, results, baseline_ms: float):
+    """File the timed candidates in the archive of kernel variants (one elite per descriptor cell; the table
+    default is every other candidate's parent) and report cells, gradients at the default's cell and
+    selection weights."""
+    from paper_2603_12440_b200 import archive
+    a = archive.Archive(capacity=64)
+    ok = [r for r in results if "ms_median" in r]
+    if not ok:
+        return None
+    parent = ok[0]
+    pc, pf = descriptors(config, parent["candidate"]), archive.fitness(True, True, baseline_ms / parent["ms_median"])
+    a.insert(pc, pf, 0)
+    for i, r in enumerate(ok[1:], 1):
+        a.insert(descriptors(config, r["candidate"]), archive.fitness(True, True, baseline_ms / r["ms_median"]), i, pc, pf, i)
+    cells = {}
+    for c in sorted({descriptors(config, r["candidate"]) for r in ok}):
+        f, i = a.cell(c)
+        cells[str(c)] = {"fitness": round(f, 4), "elite": ok[i]["candidate"], "speedup_vs_pytorch": round(baseline_ms / ok[i]["ms_median"], 3)}
+    g, gf, gr, ge = a.gradient(pc, len(ok))
+    return {"config": config, "pytorch_ms": round(baseline_ms, 5), "cells": cells, "transitions": a.transitions(),
+            "gradient_at_default": [round(v, 4) for v in g], "fitness_rate_explore": [[round(v, 4) for v in x] for x in (gf, gr, ge)],
+            "selection_weights": {str(c): round(w, 4) for c, w in a.sampling_weights(len(ok)).items()}}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--config", default="c3", choices=["c1", "c2", "c3", "c4", "c5"])
@@ -65,6 +140,7 @@ def main():
     if ok:
         best = min(ok, key=lambda r: r["ms_median"])
         print(json.dumps({"winner": best["candidate"], "ms_median": best["ms_median"], "config": args.config}))
+        print(json.dumps({"archive": file_results(args.config, results, torch_baseline_ms(args.config, args.steps))}))
 
 
 if __name__ == "__main__":

@@ -19,10 +19,11 @@ def kf():
 
 
 def test_exports_every_declared_symbol(kf):
-    header = (ROOT / "include" / "kf.h").read_text()
+    header = (ROOT / "include" / "kf.h").read_text() + (ROOT / "include" / "kf_archive.h").read_text()
     header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
     declared = set(re.findall(r"\b(kf_[a-z_0-9]+)\s*\(", header))
-    assert {"kf_linear_epilogue", "kf_linear_epilogue_rownorm", "kf_row_softmax", "kf_row_layernorm"} <= declared
+    assert {"kf_linear_epilogue", "kf_linear_epilogue_rownorm", "kf_row_softmax", "kf_row_layernorm",
+            "kf_archive_create", "kf_archive_gradient", "kf_fitness"} <= declared
     L = kf.lib()
     for name in sorted(declared):
         assert hasattr(L, name), f"libkf.so does not export {name}"
