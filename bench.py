@@ -334,6 +334,12 @@ def run_kf(args):
         live["copy_128MiB_ms"] = round(median(cms), 5)
         live["copy_128MiB_GBs"] = round(2 * cx.numel() * 2 / (median(cms) * 1e-3) / 1e9, 1)
         del cx, cy
+        # the headline operator written as plain PyTorch calls (eager: linear, GELU, layer_norm as three library
+        # kernels), the baseline the paper's speed-ups refer to; context only, not a kf path
+        import torch.nn.functional as F
+        ems, _ = time_steps(lambda: F.layer_norm(F.gelu(F.linear(d["X"], d["W"], d["bias"])), (p.N,), d["gamma"], d["beta"],
+                                                 p.eps), 20, 3, flush)
+        live["pytorch_eager_c4_ms"] = round(median(ems), 5)
 
     # ---------------------------------------------------------------- CPU baseline (oracle, rank 0, N == 1)
     cpu = None
@@ -359,7 +365,7 @@ def run_kf(args):
 
 
 # DRAM bytes per launch from ncu captures (dram__bytes_read.sum + dram__bytes_write.sum); see profiles/
-TRAFFIC = {"c4_main": 87432960}      # 52.82 MB read + 34.61 MB written (part of Y still dirty in L2 at kernel end)
+TRAFFIC = {"c4_main": 95945472}      # 54.12 MB read + 41.82 MB written (part of Y still dirty in L2 at kernel end)
 
 
 # ------------------------------------------------------------------------------------------ CPU arms
