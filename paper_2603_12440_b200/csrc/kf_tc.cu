@@ -336,16 +336,16 @@ kf_status launch_tc_linear(const void* X, long long ldx, const void* W, long lon
             done[dev] = true;
         }
     }
-    // the forms with row-norm and activation compiled in serve every CTA-pair call; the generic form
-    // serves single row blocks and runs whenever a timing switch is set
+    // the forms with row-norm and activation compiled in serve every call; the generic form runs whenever
+    // a timing switch is set
     kf_status ls;
 #ifdef KF_TC_COUNTERS                                   // build option: cycle counters in the specialised forms too
-    const bool spec = cta_group == 2 && (p.debug & ~1024) == 0;
+    const bool spec = (p.debug & ~1024) == 0;
 #else
-    const bool spec = cta_group == 2 && p.debug == 0;
+    const bool spec = p.debug == 0;
 #endif
     if (spec) {
-        const TcLaunchArgs la = {grid, st, &tmX, &tmW, &tmY, &p};
+        const TcLaunchArgs la = {cta_group, grid, st, &tmX, &tmW, &tmY, &p};
         switch (rn.norm) {
         case KF_NORM_NONE: ls = tc_launch_spec_none(ep.act, la); break;
         case KF_NORM_SOFTMAX: ls = tc_launch_spec_softmax(ep.act, la); break;

@@ -30,7 +30,7 @@
 // workspace status word, raises a CTA-wide abort flag and the CTA drains and exits.
 //
 // This header holds the kernel template; kf_tc.cu instantiates the generic form (row-norm and
-// activation read from the parameters, timing switches honoured) and kf_tc_spec*.cu the forms
+// activation read from the parameters, honoured only when a timing switch is set) and kf_tc_spec*.cu the forms
 // with both fixed at compile time, whose straight-line epilogue is a fraction of the size: the
 // epilogue code is fully unrolled over the 128 columns a thread owns, and its instruction
 // footprint, not its arithmetic, is what the generic form pays for.
@@ -635,25 +635,26 @@ kf_status tc_launch_instance(int grid, cudaStream_t st, const CUtensorMap& tmX, 
     return KF_OK;
 }
 
-// the six activations of one row-norm (CTA pairs)
-template <int NORM>
+// the six activations of one row-norm, for single CTAs (CG 1) or CTA pairs (CG 2)
+template <int CG, int NORM>
 kf_status tc_launch_norm(int act, int grid, cudaStream_t st, const CUtensorMap& tmX, const CUtensorMap& tmW,
                          const CUtensorMap& tmY, const TcParams& p) {
     switch (act) {
-    case KF_ACT_NONE: return tc_launch_instance<2, NORM, KF_ACT_NONE>(grid, st, tmX, tmW, tmY, p);
-    case KF_ACT_GELU_ERF: return tc_launch_instance<2, NORM, KF_ACT_GELU_ERF>(grid, st, tmX, tmW, tmY, p);
-    case KF_ACT_GELU_TANH: return tc_launch_instance<2, NORM, KF_ACT_GELU_TANH>(grid, st, tmX, tmW, tmY, p);
-    case KF_ACT_SILU: return tc_launch_instance<2, NORM, KF_ACT_SILU>(grid, st, tmX, tmW, tmY, p);
-    case KF_ACT_RELU: return tc_launch_instance<2, NORM, KF_ACT_RELU>(grid, st, tmX, tmW, tmY, p);
-    case KF_ACT_SIGMOID: return tc_launch_instance<2, NORM, KF_ACT_SIGMOID>(grid, st, tmX, tmW, tmY, p);
+    case KF_ACT_NONE: return tc_launch_instance<CG, NORM, KF_ACT_NONE>(grid, st, tmX, tmW, tmY, p);
+    case KF_ACT_GELU_ERF: return tc_launch_instance<CG, NORM, KF_ACT_GELU_ERF>(grid, st, tmX, tmW, tmY, p);
+    case KF_ACT_GELU_TANH: return tc_launch_instance<CG, NORM, KF_ACT_GELU_TANH>(grid, st, tmX, tmW, tmY, p);
+    case KF_ACT_SILU: return tc_launch_instance<CG, NORM, KF_ACT_SILU>(grid, st, tmX, tmW, tmY, p);
+    case KF_ACT_RELU: return tc_launch_instance<CG, NORM, KF_ACT_RELU>(grid, st, tmX, tmW, tmY, p);
+    case KF_ACT_SIGMOID: return tc_launch_instance<CG, NORM, KF_ACT_SIGMOID>(grid, st, tmX, tmW, tmY, p);
     default: return KF_ERR_INVALID_ARG;
     }
 }
 
 }  // namespace
 
-// specialised CTA-pair kernels, one translation unit per row-norm (kf_tc_spec*.cu)
+// specialised kernels, one translation unit per row-norm (kf_tc_spec*.cu)
 struct TcLaunchArgs {
+    int cta_group;              // 1 or 2
     int grid;
     cudaStream_t st;
     const CUtensorMap* tmX;

@@ -5,7 +5,9 @@
 namespace kf {
 
 kf_status tc_launch_spec_softmax(int act, const TcLaunchArgs& a) {
-    return tc_launch_norm<KF_NORM_SOFTMAX>(act, a.grid, a.st, *a.tmX, *a.tmW, *a.tmY, *static_cast<const TcParams*>(a.params));
+    const TcParams& p = *static_cast<const TcParams*>(a.params);
+    if (a.cta_group == 2) return tc_launch_norm<2, KF_NORM_SOFTMAX>(act, a.grid, a.st, *a.tmX, *a.tmW, *a.tmY, p);
+    return tc_launch_norm<1, KF_NORM_SOFTMAX>(act, a.grid, a.st, *a.tmX, *a.tmW, *a.tmY, p);
 }
 
 }  // namespace kf
