@@ -259,6 +259,22 @@ size_t tc_partials_bytes(long long M, long long N) {
     return (size_t)tm * BM * nsub * sizeof(float4);
 }
 
+// K slices per tile for a single row block with a long K: when the tiles alone leave most SMs idle, a cluster of
+// 2, 4 or 8 CTAs shares each tile's K range, as many as still fit the device.  The exchange costs two
+// cluster barriers and a second cold pass through the epilogue code, which a K below ~6000 does not
+// pay back (measured: 64 x 4096 x 4096 the same with and without, 128 x 2048 x 8192 0.059 -> 0.027 ms).
+int tc_default_splitk(long long M, long long N, long long K, int cta_group) {
+    if (cta_group != 1 || M > BM) return 1;
+    const long long tiles = (N + BN - 1) / BN, kblocks = (K + BK - 1) / BK;
+    if (kblocks < 96) return 1;
+    int sk = 1;
+    for (int c = 2; c <= 8; c *= 2) {
+        const long long per = (kblocks + c - 1) / c;       // k-blocks per slice: every slice must get at least one
+        if (tiles * c <= sm_count() && kblocks >= 2 * c && (c - 1) * per < kblocks) sk = c;
+    }
+    return sk;
+}
+
 int tc_default_grid(long long M, long long N, int cta_group) {
     const long long tm = (M + BM - 1) / BM, tn = (N + BN - 1) / BN;
     const long long units = ((tm + cta_group - 1) / cta_group) * tn;
@@ -303,9 +319,23 @@ kf_status launch_tc_linear(const void* X, long long ldx, const void* W, long lon
     }();
     p.timeout_cycles = timeout_cycles;
 
+    static const int env_sk = [] {                         // KF_TC_SPLITK=1 switches split K off; 2, 4, 8 force that many slices
+        const char* e = std::getenv("KF_TC_SPLITK");
+        return e ? std::atoi(e) : 0;
+    }();
+    p.splitk = tc_default_splitk(M, N, K, cta_group);
+    if (env_sk == 1) p.splitk = 1;
+    if ((env_sk == 2 || env_sk == 4 || env_sk == 8) && cta_group == 1 && M <= BM) {     // forced where the slices are legal
+        const long long tiles = (N + BN - 1) / BN, kblocks = (K + BK - 1) / BK, per = (kblocks + env_sk - 1) / env_sk;
+        if (tiles * env_sk <= sm_count() && kblocks >= 2 * env_sk && (env_sk - 1) * per < kblocks) p.splitk = env_sk;
+    }
     int grid = tc_default_grid(M, N, cta_group);
-    if (grid_override > 0 && grid_override < grid) grid = grid_override - grid_override % cta_group;
-    if (grid < cta_group) grid = cta_group;
+    if (p.splitk > 1) {
+        grid = (int)((N + BN - 1) / BN) * p.splitk;        // one cluster per tile, all resident at once
+    } else {
+        if (grid_override > 0 && grid_override < grid) grid = grid_override - grid_override % cta_group;
+        if (grid < cta_group) grid = cta_group;
+    }
     if (grid_out) *grid_out = grid;
     // finishing pass: one warp per row keeps the most rows in flight (measured best on C4 and C5);
     // more warps per row only for very long rows, whose coefficient table would not fit otherwise

@@ -11,6 +11,8 @@ int tc_default_cta_group(long long M, long long N);
 // bytes of per-row, per-tile partial statistics behind the status block of the workspace
 size_t tc_partials_bytes(long long M, long long N);
 int tc_default_grid(long long M, long long N, int cta_group);
+// K slices per tile (CTAs per cluster) of a single-row-block call; 1 = no split
+int tc_default_splitk(long long M, long long N, long long K, int cta_group);
 // launches the persistent GEMM (+ finishing kernel for a row-norm); all pointers 16-byte aligned,
 // K, N and every pitch multiples of 8, K >= 1
 kf_status launch_tc_linear(const void* X, long long ldx, const void* W, long long ldw, void* Y, long long ldy,

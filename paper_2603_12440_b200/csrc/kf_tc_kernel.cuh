@@ -102,6 +102,7 @@ struct TcParams {
     uint32_t* status;
     __nv_bfloat16* Y;           // output (or 16-bit intermediate), row pitch ldy
     long long ldy;
+    int splitk;                 // single CTAs only: K slices per tile = CTAs per cluster (1 = off)
     int debug;                  // generic form only; timing experiments (results are wrong): 1 no TMA loads, 2 no MMAs,
                                 // 4 no epilogue work, 8 no stores, 16 no TMEM loads, 32 no activation, 64 no residual,
                                 // 256 a longer epilogue; 128 = register stores instead of TMA stores (results right);
@@ -233,8 +234,12 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         return;                                         // (same in both CTAs of a pair: the layout is identical)
     }
     const uint32_t rank = CG == 2 ? cluster_ctarank() : 0u;       // rank 0 of a pair issues the MMAs
-    const int unit = CG == 2 ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
-    const int num_units = CG == 2 ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+    // Split K (single CTAs, few tiles): the sk CTAs of a cluster compute the same tile over one slice of K each;
+    // the partial accumulators then meet in shared memory of the CTA that owns their 32 x 128 piece (below)
+    const int sk = CG == 1 ? p.splitk : 1;
+    const uint32_t krank = (CG == 1 && sk > 1) ? cluster_ctarank() : 0u;
+    const int unit = CG == 2 ? (int)(blockIdx.x >> 1) : (int)blockIdx.x / sk;
+    const int num_units = CG == 2 ? (int)(gridDim.x >> 1) : (int)gridDim.x / sk;
     const uint32_t bar0 = base + kSmemBar;
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
@@ -250,6 +255,8 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     const int units_m = (p.tiles_m + CG - 1) / CG;
     const int num_tiles = units_m * p.tiles_n;
     const int kblocks = (p.K + BK - 1) / BK;
+    const int kb_per = (kblocks + sk - 1) / sk;           // this CTA's slice of the k-blocks (all of them without split K)
+    const int kb_begin = (int)krank * kb_per, kb_end = min(kblocks, kb_begin + kb_per);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -294,7 +301,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             for (int tile = unit; tile < num_tiles && ok; tile += num_units) {
                 if (debug & 512) break;                  // time-out test: nothing is ever loaded or signalled
                 const int mb = (tile / p.tiles_n) * CG + (int)rank, nb = tile % p.tiles_n;
-                for (int kb = 0; kb < kblocks; ++kb) {
+                for (int kb = kb_begin; kb < kb_end; ++kb) {
                     if (!mbar_wait_inl(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 0x100u + stage)) { ok = false; break; }
                     if (debug & 1) {
                         if (rank == 0) mbar_arrive(full_bar(stage));
@@ -327,7 +334,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
                 tw_acc += tick() - ta;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
-                for (int kb = 0; kb < kblocks; ++kb) {
+                for (int kb = kb_begin; kb < kb_end; ++kb) {
                     const long long tf = tick();
                     if (!mbar_wait_inl(full_bar(stage), phase, abort_flag, p.status, 0x300u + stage)) { ok = false; break; }
                     tw_full += tick() - tf;
@@ -340,7 +347,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
                         const uint64_t ad = smem_desc_sw128(a_addr + k * UMMA_K * 2);
                         const uint64_t bd = smem_desc_sw128(b_addr + k * UMMA_K * 2);
                         if (CG == 2) tc_mma_bf16_pair(d_tmem, ad, bd, kIdesc<2>, (kb | k) != 0 ? 1u : 0u);
-                        else tc_mma_bf16(d_tmem, ad, bd, kIdesc<1>, (kb | k) != 0 ? 1u : 0u);
+                        else tc_mma_bf16(d_tmem, ad, bd, kIdesc<1>, ((kb - kb_begin) | k) != 0 ? 1u : 0u);
                     }
                     // stage reusable (in both CTAs of a pair) once these MMAs have read it
                     if (CG == 2) {
@@ -369,6 +376,11 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             }
         }
       }
+      if (CG == 1 && sk > 1) {                             // the two cluster barriers of the split-K exchange (epilogue warps)
+          __syncwarp();
+          cluster_sync_all();
+          cluster_sync_all();
+      }
     } else {
         reg_alloc<kRegsEpi>();
         // ------------------------------------------------------------------ epilogue warps
@@ -378,6 +390,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         uint32_t acc = 0, acc_phase = 0, it = 0, nstore = 0;
         const uint32_t stage_base = base + kSmemStage + (uint32_t)(warp - kRoleWarps) * 2u * kStageBufBytes;
         bool ok = true;
+        bool sk_synced = false;
         long long te_wait = 0, te_work = 0, te_s1 = 0;
         for (int tile = unit; tile < num_tiles && ok; tile += num_units, ++it) {
             const long long te0 = tick();
@@ -422,6 +435,51 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
                 else mbar_arrive(tempty_bar(acc));
             }
             te_s1 += tick() - te1;
+
+            bool owner = true;
+            if (CG == 1 && sk > 1) {
+                // Split K: the eight 32 x 128 pieces of the tile (one per epilogue warp) are dealt round the
+                // cluster; every CTA writes its partial of a piece it does not own into the owner's idle
+                // operand ring ([piece][sender][16-byte vector][lane]: the same lane-contiguous layout
+                // for writer and reader, free of bank conflicts), the owner adds the partials to its
+                // own in sender order and runs the epilogue of the piece.
+                cluster_sync_all();                         // every CTA of the cluster is done with its operand ring
+                const int slot = warp - kRoleWarps;
+                const uint32_t own_rank = (uint32_t)(slot % sk);
+                const uint32_t piece_bytes = 32u * 32u * 16u;
+                owner = own_rank == krank;
+                if (!owner && ok) {
+                    const uint32_t sidx = krank < own_rank ? krank : krank - 1u;
+                    const uint32_t dst = map_to_cta(base + ((uint32_t)(slot / sk) * (uint32_t)(sk - 1) + sidx) * piece_bytes +
+                                                        (uint32_t)lane * 16u, own_rank);
+#pragma unroll
+                    for (int c = 0; c < kSub / 32; ++c)
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            st_cluster_v4(dst + (uint32_t)(c * 8 + j) * 512u, v[c][4 * j], v[c][4 * j + 1], v[c][4 * j + 2],
+                                          v[c][4 * j + 3]);
+                }
+                cluster_sync_all();                         // the partials have landed (release / acquire)
+                sk_synced = true;
+                if (owner) {
+                    for (int sdr = 0; sdr < sk - 1; ++sdr) {
+                        const uint32_t src = base + ((uint32_t)(slot / sk) * (uint32_t)(sk - 1) + (uint32_t)sdr) * piece_bytes +
+                                             (uint32_t)lane * 16u;
+#pragma unroll
+                        for (int c = 0; c < kSub / 32; ++c)
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                uint32_t a0, a1, a2, a3;
+                                ld_shared_v4(src + (uint32_t)(c * 8 + j) * 512u, a0, a1, a2, a3);
+                                v[c][4 * j] = __float_as_uint(__uint_as_float(v[c][4 * j]) + __uint_as_float(a0));
+                                v[c][4 * j + 1] = __float_as_uint(__uint_as_float(v[c][4 * j + 1]) + __uint_as_float(a1));
+                                v[c][4 * j + 2] = __float_as_uint(__uint_as_float(v[c][4 * j + 2]) + __uint_as_float(a2));
+                                v[c][4 * j + 3] = __float_as_uint(__uint_as_float(v[c][4 * j + 3]) + __uint_as_float(a3));
+                            }
+                    }
+                }
+            }
+            if (owner) {
 
             // element-wise epilogue in place on column pairs, per-row statistics of the sub-tile; columns
             // beyond N (ragged last chunk) are set to the neutral value of the statistic
@@ -555,8 +613,13 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             if (norm != KF_NORM_NONE && row_ok && nchunks > 0)
                 p.partials[((size_t)mb * BM + q * 32 + lane) * p.nsub + (nb * 2 + half)] =
                     make_float4(st_shift, st_s1, st_s2, st_scale);
+            }                                               // owner of the piece
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
             te_work += tick() - te1;
+        }
+        if (CG == 1 && sk > 1 && !sk_synced) {               // gave up before the exchange: the cluster still counts this warp in
+            cluster_sync_all();
+            cluster_sync_all();
         }
         if (lane == 0) tma_store_wait_all<0>();              // the staging buffers are read, Y is written
         if (count_on && warp == kRoleWarps && lane == 0) {
@@ -623,7 +686,7 @@ kf_status tc_launch_instance(int grid, cudaStream_t st, const CUtensorMap& tmX, 
     lc.stream = st;
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeClusterDimension;
-    at[0].val.clusterDim.x = CG;
+    at[0].val.clusterDim.x = CG == 2 ? 2 : (p.splitk > 1 ? p.splitk : 1);
     at[0].val.clusterDim.y = 1;
     at[0].val.clusterDim.z = 1;
     lc.attrs = at;

@@ -170,6 +170,19 @@ def test_tc_tall_and_very_wide_rownorm(kf, M, N, K, norm):
     assert_parity(run(kf, p), oracle_of(p), "bf16", f"{norm} {M}x{N}x{K}")
 
 
+@pytest.mark.parametrize("M,N,K,norm", [(128, 2056, 8200, "layernorm"),      # 9 tiles x 8 K slices
+                                         (70, 9480, 6160, "softmax"),          # 38 tiles x 2 slices, ragged everywhere
+                                         (1, 520, 12296, "none")])             # 3 tiles x 8 slices, one row
+def test_tc_split_k_single_row_block(kf, M, N, K, norm):
+    """One row block and a long K: the K range of a tile is shared by the CTAs of a cluster and the partial
+    accumulators are added in the owner's shared memory before the epilogue."""
+    p = make("bf16", M, N, K, seed=71 + M, act="gelu_erf", norm=norm, res=True)
+    assert kf.tile_config(M, N, K, torch.bfloat16, norm)["cta_group"] == 1
+    got = run(kf, p)
+    assert_parity(got, oracle_of(p), "bf16", f"split-K {norm} {M}x{N}x{K}")
+    assert np.array_equal(got, run(kf, p))                  # fixed summation order: the same bits every time
+
+
 def test_tc_layernorm_with_mean_far_from_zero(kf):
     # sigmoid outputs sit near 0.5 with a small spread: the per-tile shift keeps the deviations exact
     p = make("bf16", 200, 1536, 256, seed=27, act="sigmoid", norm="layernorm", res=False, std=0.01)

@@ -16,8 +16,9 @@ import sys
 sys.path.insert(0, %r)
 import torch
 import paper_2603_12440_b200 as kf
-x = torch.randn(300, 256, device="cuda", dtype=torch.bfloat16)
-w = torch.randn(520, 256, device="cuda", dtype=torch.bfloat16)
+M, N, K = [int(v) for v in sys.argv[1:4]]
+x = torch.randn(M, K, device="cuda", dtype=torch.bfloat16)
+w = torch.randn(N, K, device="cuda", dtype=torch.bfloat16)
 y = kf.linear_epilogue_rownorm(x, w, norm="softmax")
 try:
     kf.check_device_status()
@@ -33,9 +34,12 @@ print("ROWSUM", float(z.sum(1).mean()))
 
 
 @pytest.mark.gpu
-def test_bounded_waits_report_a_timeout_and_the_context_survives():
+@pytest.mark.parametrize("shape", [(300, 520, 256),        # CTA pairs
+                                   (64, 520, 8192)])       # one row block, K shared by a cluster of eight CTAs: every
+def test_bounded_waits_report_a_timeout_and_the_context_survives(shape):   # warp still meets the cluster barriers
     env = dict(os.environ, KF_TC_DEBUG="512", KF_TC_TIMEOUT_MS="150")
-    out = subprocess.run([sys.executable, "-c", CHILD % str(ROOT)], env=env, capture_output=True, text=True, timeout=240)
+    out = subprocess.run([sys.executable, "-c", CHILD % str(ROOT), *[str(v) for v in shape]], env=env, capture_output=True,
+                         text=True, timeout=240)
     assert out.returncode == 0, out.stderr[-2000:]
     lines = out.stdout.strip().splitlines()
     assert "STATUS 6" in lines, out.stdout          # KF_ERR_TIMEOUT
