@@ -279,7 +279,11 @@ int tc_default_grid(long long M, long long N, int cta_group) {
     const long long tm = (M + BM - 1) / BM, tn = (N + BN - 1) / BN;
     const long long units = ((tm + cta_group - 1) / cta_group) * tn;
     const long long slots = sm_count() / cta_group;
-    return (int)((units < slots ? units : slots) * cta_group);
+    if (units <= slots) return (int)(units * cta_group);
+    // the number of rounds is fixed by the device; the fewest CTAs that still finish in that many rounds share
+    // the work evenly, and the SMs left out leave their share of the power budget to the others
+    const long long rounds = (units + slots - 1) / slots;
+    return (int)(((units + rounds - 1) / rounds) * cta_group);
 }
 
 kf_status launch_tc_linear(const void* X, long long ldx, const void* W, long long ldw, void* Y, long long ldy,
