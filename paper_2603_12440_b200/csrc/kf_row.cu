@@ -182,17 +182,22 @@ __device__ __forceinline__ void bulk_load_row(uint32_t dst, const void* src, uin
                  : "memory");
 }
 
-template <typename T, int NORM, int VPT>
-__global__ void __launch_bounds__(kRingThreads, 1)
-row_norm_ring_kernel(const T* X, long long ldx, T* Y, long long ldy, long long M, int N, int slots,
+// CONS consumer warps (16 for rows of 8 KiB, 28 where that many slots fit: short rows are bound by the latency of
+// a row's passes and reductions, which more warps hide); BATCH: a slot holds rb > 1 rows
+template <typename T, int NORM, int VPT, int CONS, bool BATCH>
+__global__ void __launch_bounds__(32 * (CONS + 1), 1)
+row_norm_ring_kernel(const T* X, long long ldx, T* Y, long long ldy, long long M, int N, int slots, int rb,
                      const T* __restrict__ gamma, const T* __restrict__ beta, float eps) {
     constexpr int E = Elem<T>::kVec;
     extern __shared__ __align__(128) uint8_t ring_smem[];
     const int NV = N / E;
     const uint32_t row_bytes = (uint32_t)N * sizeof(T);
-    // layout: [slots x row_bytes][gamma lo/hi float4 arrays][beta lo/hi float4 arrays][barriers]
+    // A slot holds a block of rb consecutive rows (short rows travel several to a copy and a barrier round).
+    // layout: [slots x rb x row_bytes][gamma lo/hi float4 arrays][beta lo/hi float4 arrays][barriers]
+    if (!BATCH) rb = 1;                                  // (folds every use below to the one-row form)
+    const uint32_t slot_bytes = (uint32_t)rb * row_bytes;
     uint8_t* ring = ring_smem;
-    float4* gam = reinterpret_cast<float4*>(ring_smem + (size_t)slots * row_bytes);
+    float4* gam = reinterpret_cast<float4*>(ring_smem + (size_t)slots * slot_bytes);
     float4* bet = gam + (NORM == KF_NORM_SOFTMAX ? 0 : (E / 4) * NV);
     uint64_t* bars = reinterpret_cast<uint64_t*>(bet + (NORM == KF_NORM_LAYERNORM ? (E / 4) * NV : 0));
     const uint32_t bar0 = smem_addr(bars);
@@ -209,18 +214,26 @@ row_norm_ring_kernel(const T* X, long long ldx, T* Y, long long ldy, long long M
     }
     __syncthreads();                                     // barriers exist; the producer starts at once
 
-    // rows of this CTA: blockIdx.x, blockIdx.x + gridDim.x, ...; its i-th row uses slot i % slots
-    const long long my_rows = (M - blockIdx.x + gridDim.x - 1) / gridDim.x;
+    // row blocks of this CTA: blockIdx.x, blockIdx.x + gridDim.x, ...; its i-th block uses slot i % slots
+    const long long nblocks = (M + rb - 1) / rb;
+    const long long my_rows = (nblocks - blockIdx.x + gridDim.x - 1) / gridDim.x;
 
-    if (warp == kRingConsumers) {
+    if (warp == CONS) {
         if (lane == 0) {
             for (long long i = 0; i < my_rows; ++i) {
                 const int s = (int)(i % slots);
                 const uint32_t ph = (uint32_t)((i / slots) & 1);
                 if (!rbar_wait(empty_bar(s), ph ^ 1u)) break;
-                rbar_expect_tx(full_bar(s), row_bytes);
-                const long long row = blockIdx.x + i * (long long)gridDim.x;
-                bulk_load_row(smem_addr(ring + (size_t)s * row_bytes), X + row * ldx, row_bytes, full_bar(s));
+                const long long row0 = (blockIdx.x + i * (long long)gridDim.x) * rb;
+                const int nrows = (int)((M - row0 < rb) ? M - row0 : rb);
+                rbar_expect_tx(full_bar(s), (uint32_t)nrows * row_bytes);
+                const uint32_t dst = smem_addr(ring + (size_t)s * slot_bytes);
+                if (!BATCH || ldx == N) {                    // one row, or a contiguous block: one copy
+                    bulk_load_row(dst, X + row0 * ldx, (uint32_t)nrows * row_bytes, full_bar(s));
+                } else {
+                    for (int r = 0; r < nrows; ++r)
+                        bulk_load_row(dst + (uint32_t)r * row_bytes, X + (row0 + r) * ldx, row_bytes, full_bar(s));
+                }
             }
         }
         return;
@@ -229,7 +242,7 @@ row_norm_ring_kernel(const T* X, long long ldx, T* Y, long long ldy, long long M
     // consumers, while the first rows are in flight: gamma / beta as fp32, de-interleaved so that a
     // lane's two float4 halves are conflict-free reads; then a barrier among the consumer warps only
     if (NORM != KF_NORM_SOFTMAX) {
-        for (int idx = threadIdx.x; idx < NV; idx += kRingConsumers * 32) {
+        for (int idx = threadIdx.x; idx < NV; idx += CONS * 32) {
             float g[E], b[E];
 #pragma unroll
             for (int e = 0; e < E; ++e) { g[e] = 1.f; b[e] = 0.f; }
@@ -242,15 +255,18 @@ row_norm_ring_kernel(const T* X, long long ldx, T* Y, long long ldy, long long M
                     bet[h * NV + idx] = make_float4(b[h * 4], b[h * 4 + 1], b[h * 4 + 2], b[h * 4 + 3]);
             }
         }
-        asm volatile("bar.sync 1, %0;" ::"n"(kRingConsumers * 32) : "memory");
+        asm volatile("bar.sync 1, %0;" ::"n"(CONS * 32) : "memory");
     }
 
-    for (long long i = warp; i < my_rows; i += kRingConsumers) {
+    for (long long i = warp; i < my_rows; i += CONS) {
         const int s = (int)(i % slots);
         const uint32_t ph = (uint32_t)((i / slots) & 1);
-        const long long row = blockIdx.x + i * (long long)gridDim.x;
+        const long long row0 = (blockIdx.x + i * (long long)gridDim.x) * rb;
+        const int nrows = (int)((M - row0 < rb) ? M - row0 : rb);
         if (!rbar_wait(full_bar(s), ph)) break;
-        const uint4* srow = reinterpret_cast<const uint4*>(ring + (size_t)s * row_bytes);
+        for (int r = 0; r < (BATCH ? nrows : 1); ++r) {
+        const long long row = row0 + r;
+        const uint4* srow = reinterpret_cast<const uint4*>(ring + (size_t)s * slot_bytes + (size_t)r * row_bytes);
         uint4* yr = reinterpret_cast<uint4*>(Y + row * ldy);
         // The row stays in shared memory and is swept twice (statistics, then output), so a warp needs
         // few registers and many warps fit: latency is hidden by warps, not by a register-resident row.
@@ -327,6 +343,7 @@ row_norm_ring_kernel(const T* X, long long ldx, T* Y, long long ldy, long long M
                 }
             }
         }
+        }                                                   // rows of the block
         __syncwarp();
         if (lane == 0) rbar_arrive(empty_bar(s));           // every lane has finished reading the slot
     }
@@ -420,36 +437,58 @@ cudaError_t launch_typed(const void* X, long long ldx, void* Y, long long ldy, l
         const size_t row_bytes = (size_t)N * sizeof(T);
         const size_t vec_bytes = (NORM == KF_NORM_SOFTMAX ? 0 : (NORM == KF_NORM_LAYERNORM ? 2 : 1)) * (size_t)N * 4;
         const size_t budget = 226 * 1024;
-        long long slots = ((long long)budget - (long long)vec_bytes - 64) / (long long)(row_bytes + 16);
-        // a slot must always come back to the same consumer warp (row i -> slot i % slots, warp
+        // rows per slot: short rows are batched up to 8 KiB a slot, as long as every CTA still gets
+        // a few slots' worth of blocks
+        int rb = 1;
+        while (rb < 32 && (size_t)(2 * rb) * row_bytes <= 8192 && M / (2 * rb) >= 8ll * sms) rb <<= 1;
+        static const int env_rb = [] {
+            const char* e = std::getenv("KF_ROW_RB");
+            return e ? std::atoi(e) : 0;
+        }();
+        if (env_rb >= 1 && env_rb <= 64 && (size_t)env_rb * row_bytes <= 16384) rb = env_rb;
+        const size_t slot_bytes = (size_t)rb * row_bytes;
+        long long slots = ((long long)budget - (long long)vec_bytes - 64) / (long long)(slot_bytes + 16);
+        // 28 consumer warps where that many slots fit the shared memory (rows up to 4 KiB), else 16
+        const bool many = (long long)(28 * (slot_bytes + 16) + vec_bytes + 64) <= (long long)budget && vpt <= 8;
+        const int cons = many ? 28 : kRingConsumers;
+        // a slot must always come back to the same consumer warp (block i -> slot i % slots, warp
         // i % consumers): then a warp only ever waits for the phase right after one it consumed itself
-        slots -= slots % kRingConsumers;
-        if (slots > 4 * kRingConsumers) slots = 4 * kRingConsumers;
-        if (slots >= kRingConsumers) {
-            const size_t smem = slots * row_bytes + vec_bytes + 2 * slots * 8;
-            const int grid = (int)(M < sms ? M : sms);
+        slots -= slots % cons;
+        if (slots > 4 * cons) slots = 4 * cons;
+        if (slots >= cons) {
+            const size_t smem = slots * slot_bytes + vec_bytes + 2 * slots * 8;
+            const long long nblocks = (M + rb - 1) / rb;
+            const int grid = (int)(nblocks < sms ? nblocks : sms);
             cudaError_t e = cudaSuccess;
-#define KF_RING_LAUNCH(V)                                                                                      \
+#define KF_RING_LAUNCH_K(V, C, B)                                                                              \
     do {                                                                                                       \
         static bool attr_done[64] = {};                                                                        \
         int dev = 0;                                                                                           \
         cudaGetDevice(&dev);                                                                                   \
         if (dev >= 0 && dev < 64 && !attr_done[dev]) {                                                         \
-            e = cudaFuncSetAttribute(row_norm_ring_kernel<T, NORM, V>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                                     226 * 1024);                                                              \
+            e = cudaFuncSetAttribute(row_norm_ring_kernel<T, NORM, V, C, B>,                                   \
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024);                 \
             attr_done[dev] = e == cudaSuccess;                                                                 \
         }                                                                                                      \
         if (e == cudaSuccess)                                                                                  \
-            row_norm_ring_kernel<T, NORM, V><<<grid, kRingThreads, smem, st>>>(x, ldx, y, ldy, M, (int)N,      \
-                                                                               (int)slots, g, b, rn.eps);      \
+            row_norm_ring_kernel<T, NORM, V, C, B><<<grid, 32 * (C + 1), smem, st>>>(x, ldx, y, ldy, M, (int)N, \
+                                                                                     (int)slots, rb, g, b, rn.eps); \
+    } while (0)
+#define KF_RING_LAUNCH(V)                                                                                      \
+    do {                                                                                                       \
+        if (many && rb > 1) KF_RING_LAUNCH_K(V, 28, true);                                                     \
+        else if (many) KF_RING_LAUNCH_K(V, 28, false);                                                         \
+        else if (rb > 1) KF_RING_LAUNCH_K(V, kRingConsumers, true);                                            \
+        else KF_RING_LAUNCH_K(V, kRingConsumers, false);                                                       \
     } while (0)
             switch (vpt) {
             case 1: KF_RING_LAUNCH(1); break;
             case 2: KF_RING_LAUNCH(2); break;
             case 4: KF_RING_LAUNCH(4); break;
             case 8: KF_RING_LAUNCH(8); break;
-            default: KF_RING_LAUNCH(16); break;
+            default: KF_RING_LAUNCH_K(16, kRingConsumers, false); break;
             }
+#undef KF_RING_LAUNCH_K
 #undef KF_RING_LAUNCH
             if (e != cudaSuccess) return e;
             return cudaGetLastError();
