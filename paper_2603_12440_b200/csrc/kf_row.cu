@@ -3,7 +3,7 @@
 // Fast path: a row lives in the registers of TPR threads as VPT 16-byte vectors each, so every
 // element is read from HBM once and written once (streaming loads/stores, 128-bit, coalesced);
 // statistics use warp shuffles, plus one shared-memory hop when a row spans several warps.
-// LayerNorm takes the mean first and the centred sum of squares second, both from registers.
+// LayerNorm takes both moments in one sweep about a shift from the row itself (one reduction round).
 // Generic path (row length or pointers not 16-byte friendly, or rows too long for registers):
 // one CTA per row, scalar accesses, three passes over global memory.
 #include "kf_common.cuh"
@@ -32,13 +32,29 @@ __device__ __forceinline__ float group_reduce(float v, int tpr, float* red) {
     for (int i = 1; i < wpg; ++i) t = IS_MAX ? fmaxf(t, red[g0 + i]) : t + red[g0 + i];
     return t;
 }
+// two sums at once, one barrier round: `red2` has two floats per warp of the CTA
+__device__ __forceinline__ float2 group_sum2(float a, float b, int tpr, float2* red2) {
+    a = warp_sum(a);
+    b = warp_sum(b);
+    if (tpr <= 32) return make_float2(a, b);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int wpg = tpr >> 5, g0 = (warp / wpg) * wpg;
+    __syncthreads();
+    if (lane == 0) red2[warp] = make_float2(a, b);
+    __syncthreads();
+    float2 t = red2[g0];
+    for (int i = 1; i < wpg; ++i) { t.x += red2[g0 + i].x; t.y += red2[g0 + i].y; }
+    return t;
+}
 
+// (up to eight vectors a thread the kernel is held to 64 registers: the bytes in flight come from occupancy here)
 template <typename T, int NORM, int VPT>
-__global__ void __launch_bounds__(512)
+__global__ void __launch_bounds__(512, VPT <= 8 ? 2 : 1)
 row_norm_reg_kernel(const T* X, long long ldx, T* Y, long long ldy, long long M,   // Y may alias X
                     int N, int tpr, const T* __restrict__ gamma, const T* __restrict__ beta, float eps) {
     constexpr int E = Elem<T>::kVec;
     __shared__ float red[32];
+    __shared__ float2 red2[32];
     const int rows_per_cta = blockDim.x / tpr;
     const long long row = (long long)blockIdx.x * rows_per_cta + threadIdx.x / tpr;
     const int lr = threadIdx.x % tpr;
@@ -86,27 +102,28 @@ row_norm_reg_kernel(const T* X, long long ldx, T* Y, long long ldy, long long M,
             }
         }
     } else {
-        float mean = 0.f;
-        if (NORM == KF_NORM_LAYERNORM) {
-            float s = 0.f;
-#pragma unroll
-            for (int i = 0; i < VPT; ++i)
-                if (lr + i * tpr < NV) {
-                    unpack<T>(v[i], f);
-#pragma unroll
-                    for (int e = 0; e < E; ++e) s += f[e];
-                }
-            mean = group_reduce<false>(s, tpr, red) / (float)N;
-        }
-        float q = 0.f;
+        // both moments in one sweep and one reduction round, about a shift c taken from the row itself (its first
+        // element, read by every thread of the row): sum(x - c) and sum((x - c)^2) lose nothing to cancellation
+        // because c lies inside the data; RMSNorm: c = 0
+        float c = 0.f;
+        if (NORM == KF_NORM_LAYERNORM && live) c = Elem<T>::load(X + row * ldx);
+        float a = 0.f, q = 0.f;
 #pragma unroll
         for (int i = 0; i < VPT; ++i)
             if (lr + i * tpr < NV) {
                 unpack<T>(v[i], f);
 #pragma unroll
-                for (int e = 0; e < E; ++e) { const float d = f[e] - mean; q = fmaf(d, d, q); }
+                for (int e = 0; e < E; ++e) { const float d = f[e] - c; a += d; q = fmaf(d, d, q); }
             }
-        q = group_reduce<false>(q, tpr, red);
+        float mean = 0.f;
+        if (NORM == KF_NORM_LAYERNORM) {
+            const float2 sq = group_sum2(a, q, tpr, red2);
+            const float dm = sq.x / (float)N;
+            mean = c + dm;
+            q = fmaxf(sq.y - sq.x * dm, 0.f);              // centred sum of squares
+        } else {
+            q = group_reduce<false>(q, tpr, red);
+        }
         const float rstd = rsqrtf(q / (float)N + eps);
         const uint4* gv = reinterpret_cast<const uint4*>(gamma);
         const uint4* bv = reinterpret_cast<const uint4*>(beta);
