@@ -15,6 +15,12 @@ namespace {
 
 constexpr int kRowThreads = 256;
 
+// The arithmetic below runs on pairs of neighbouring elements with the packed fp32 instructions of sm_100
+// (add / mul / fma on two floats at once): the row kernels sit close enough to the issue limit for the halved
+// instruction count to show (long LayerNorm rows most of all).
+__device__ __forceinline__ float2 pr2(const float* f, int k) { return make_float2(f[2 * k], f[2 * k + 1]); }
+__device__ __forceinline__ float2 dup2(float x) { return make_float2(x, x); }
+
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) { return __ldcs(p); }
 __device__ __forceinline__ void st_stream(uint4* p, const uint4& v) { __stcs(p, v); }
 
@@ -81,23 +87,31 @@ row_norm_reg_kernel(const T* X, long long ldx, T* Y, long long ldy, long long M,
             }
         m = group_reduce<true>(m, tpr, red);
         const float ms = m * kLog2e;
-        float s = 0.f;
+        const float2 l2e = dup2(kLog2e), nms = dup2(-ms);
+        float2 s2 = dup2(0.f);
 #pragma unroll
         for (int i = 0; i < VPT; ++i)
             if (lr + i * tpr < NV) {
                 unpack<T>(v[i], f);
 #pragma unroll
-                for (int e = 0; e < E; ++e) s += fast_ex2(fmaf(f[e], kLog2e, -ms));
+                for (int k = 0; k < E / 2; ++k) {
+                    const float2 t = __ffma2_rn(pr2(f, k), l2e, nms);
+                    s2 = __fadd2_rn(s2, make_float2(fast_ex2(t.x), fast_ex2(t.y)));
+                }
             }
-        s = group_reduce<false>(s, tpr, red);
-        const float inv = 1.0f / s;
+        const float s = group_reduce<false>(s2.x + s2.y, tpr, red);
+        const float2 inv = dup2(1.0f / s);
 #pragma unroll
         for (int i = 0; i < VPT; ++i) {
             const int idx = lr + i * tpr;
             if (live && idx < NV) {
                 unpack<T>(v[i], f);
 #pragma unroll
-                for (int e = 0; e < E; ++e) f[e] = fast_ex2(fmaf(f[e], kLog2e, -ms)) * inv;
+                for (int k = 0; k < E / 2; ++k) {
+                    const float2 t = __ffma2_rn(pr2(f, k), l2e, nms);
+                    const float2 o = __fmul2_rn(make_float2(fast_ex2(t.x), fast_ex2(t.y)), inv);
+                    f[2 * k] = o.x; f[2 * k + 1] = o.y;
+                }
                 st_stream(yr + idx, pack<T>(f));
             }
         }
@@ -107,14 +121,20 @@ row_norm_reg_kernel(const T* X, long long ldx, T* Y, long long ldy, long long M,
         // because c lies inside the data; RMSNorm: c = 0
         float c = 0.f;
         if (NORM == KF_NORM_LAYERNORM && live) c = Elem<T>::load(X + row * ldx);
-        float a = 0.f, q = 0.f;
+        float2 a2 = dup2(0.f), q2 = dup2(0.f);
+        const float2 nc = dup2(-c);
 #pragma unroll
         for (int i = 0; i < VPT; ++i)
             if (lr + i * tpr < NV) {
                 unpack<T>(v[i], f);
 #pragma unroll
-                for (int e = 0; e < E; ++e) { const float d = f[e] - c; a += d; q = fmaf(d, d, q); }
+                for (int k = 0; k < E / 2; ++k) {
+                    const float2 d = __fadd2_rn(pr2(f, k), nc);
+                    a2 = __fadd2_rn(a2, d);
+                    q2 = __ffma2_rn(d, d, q2);
+                }
             }
+        float a = a2.x + a2.y, q = q2.x + q2.y;
         float mean = 0.f;
         if (NORM == KF_NORM_LAYERNORM) {
             const float2 sq = group_sum2(a, q, tpr, red2);
@@ -125,6 +145,7 @@ row_norm_reg_kernel(const T* X, long long ldx, T* Y, long long ldy, long long M,
             q = group_reduce<false>(q, tpr, red);
         }
         const float rstd = rsqrtf(q / (float)N + eps);
+        const float2 rs2 = dup2(rstd), ofs2 = dup2(-mean * rstd);
         const uint4* gv = reinterpret_cast<const uint4*>(gamma);
         const uint4* bv = reinterpret_cast<const uint4*>(beta);
 #pragma unroll
@@ -136,11 +157,11 @@ row_norm_reg_kernel(const T* X, long long ldx, T* Y, long long ldy, long long M,
                 if (gamma) unpack<T>(__ldg(gv + idx), g);
                 if (beta && NORM == KF_NORM_LAYERNORM) unpack<T>(__ldg(bv + idx), b);
 #pragma unroll
-                for (int e = 0; e < E; ++e) {
-                    float o = (f[e] - mean) * rstd;
-                    if (gamma) o *= g[e];
-                    if (beta && NORM == KF_NORM_LAYERNORM) o += b[e];
-                    f[e] = o;
+                for (int k = 0; k < E / 2; ++k) {
+                    float2 o = __ffma2_rn(pr2(f, k), rs2, ofs2);     // (x - mean) * rstd
+                    if (gamma) o = __fmul2_rn(o, pr2(g, k));
+                    if (beta && NORM == KF_NORM_LAYERNORM) o = __fadd2_rn(o, pr2(b, k));
+                    f[2 * k] = o.x; f[2 * k + 1] = o.y;
                 }
                 st_stream(yr + idx, pack<T>(f));
             }
@@ -298,22 +319,30 @@ row_norm_ring_kernel(const T* X, long long ldx, T* Y, long long ldy, long long M
                     for (int e = 0; e < E; ++e) m[e & 3] = fmaxf(m[e & 3], x[e]);
                 }
             const float ms = warp_max(fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3]))) * kLog2e;
-            float l[4] = {0.f, 0.f, 0.f, 0.f};
+            const float2 l2e = dup2(kLog2e), nms = dup2(-ms);
+            float2 l[2] = {dup2(0.f), dup2(0.f)};
 #pragma unroll
             for (int v = 0; v < VPT; ++v)
                 if (lane + v * 32 < NV) {
                     unpack<T>(srow[lane + v * 32], x);
 #pragma unroll
-                    for (int e = 0; e < E; ++e) l[e & 3] += fast_ex2(fmaf(x[e], kLog2e, -ms));
+                    for (int k = 0; k < E / 2; ++k) {
+                        const float2 t = __ffma2_rn(pr2(x, k), l2e, nms);
+                        l[k & 1] = __fadd2_rn(l[k & 1], make_float2(fast_ex2(t.x), fast_ex2(t.y)));
+                    }
                 }
-            const float inv = 1.0f / warp_sum((l[0] + l[1]) + (l[2] + l[3]));
+            const float2 inv = dup2(1.0f / warp_sum((l[0].x + l[0].y) + (l[1].x + l[1].y)));
 #pragma unroll
             for (int v = 0; v < VPT; ++v) {
                 const int idx = lane + v * 32;
                 if (idx < NV) {
                     unpack<T>(srow[idx], x);
 #pragma unroll
-                    for (int e = 0; e < E; ++e) x[e] = fast_ex2(fmaf(x[e], kLog2e, -ms)) * inv;
+                    for (int k = 0; k < E / 2; ++k) {
+                        const float2 t = __ffma2_rn(pr2(x, k), l2e, nms);
+                        const float2 o = __fmul2_rn(make_float2(fast_ex2(t.x), fast_ex2(t.y)), inv);
+                        x[2 * k] = o.x; x[2 * k + 1] = o.y;
+                    }
                     st_stream(yr + idx, pack<T>(x));
                 }
             }
@@ -321,20 +350,21 @@ row_norm_ring_kernel(const T* X, long long ldx, T* Y, long long ldy, long long M
             // one sweep for both moments about a shift taken from the row itself (its first element):
             // sum(x - c) and sum((x - c)^2) lose no accuracy to cancellation because c lies inside the data
             const float c = (NORM == KF_NORM_LAYERNORM) ? Elem<T>::load(reinterpret_cast<const T*>(srow)) : 0.f;
-            float a[4] = {0.f, 0.f, 0.f, 0.f}, q[4] = {0.f, 0.f, 0.f, 0.f};
+            float2 a[2] = {dup2(0.f), dup2(0.f)}, q[2] = {dup2(0.f), dup2(0.f)};
+            const float2 nc = dup2(-c);
 #pragma unroll
             for (int v = 0; v < VPT; ++v)
                 if (lane + v * 32 < NV) {
                     unpack<T>(srow[lane + v * 32], x);
 #pragma unroll
-                    for (int e = 0; e < E; ++e) {
-                        const float d = x[e] - c;
-                        a[e & 3] += d;
-                        q[e & 3] = fmaf(d, d, q[e & 3]);
+                    for (int k = 0; k < E / 2; ++k) {
+                        const float2 d = __fadd2_rn(pr2(x, k), nc);
+                        a[k & 1] = __fadd2_rn(a[k & 1], d);
+                        q[k & 1] = __ffma2_rn(d, d, q[k & 1]);
                     }
                 }
-            const float s1 = warp_sum((a[0] + a[1]) + (a[2] + a[3]));
-            const float s2 = warp_sum((q[0] + q[1]) + (q[2] + q[3]));
+            const float s1 = warp_sum((a[0].x + a[0].y) + (a[1].x + a[1].y));
+            const float s2 = warp_sum((q[0].x + q[0].y) + (q[1].x + q[1].y));
             const float dm = (NORM == KF_NORM_LAYERNORM) ? s1 / (float)N : 0.f;      // mean - c
             const float var = fmaxf(s2 / (float)N - dm * dm, 0.f);
             const float rstd = rsqrtf(var + eps);
