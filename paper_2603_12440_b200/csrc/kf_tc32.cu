@@ -99,6 +99,7 @@ struct Tc32Params {
 };
 
 // element-wise epilogue on 32 consecutive columns of one row, accurate fp32 forms
+template <int ACT>
 __device__ __forceinline__ void epilogue32_f32(float (&a)[32], const Tc32Params& p, const float* bias32, long long row,
                                                int col0, bool row_ok) {
     if (bias32) {
@@ -109,9 +110,9 @@ __device__ __forceinline__ void epilogue32_f32(float (&a)[32], const Tc32Params&
             a[q * 4 + 0] += b.x; a[q * 4 + 1] += b.y; a[q * 4 + 2] += b.z; a[q * 4 + 3] += b.w;
         }
     }
-    if (p.act != KF_ACT_NONE) {
+    if (ACT != KF_ACT_NONE) {
 #pragma unroll
-        for (int e = 0; e < 32; ++e) a[e] = apply_act<true>(p.act, a[e]);
+        for (int e = 0; e < 32; ++e) a[e] = apply_act<true>(ACT, a[e]);
     }
     if (p.scale != 1.0f) {
 #pragma unroll
@@ -129,6 +130,9 @@ __device__ __forceinline__ void epilogue32_f32(float (&a)[32], const Tc32Params&
     }
 }
 
+// ACT: the activation compiled in (the accurate forms are long; with all six behind a run-time switch in the
+// unrolled epilogue the kernel spent five times its main loop fetching instructions)
+template <int ACT>
 __global__ void __launch_bounds__(kThreads, 1)
 tc32_linear_kernel(const __grid_constant__ CUtensorMap tmXh, const __grid_constant__ CUtensorMap tmXl,
                    const __grid_constant__ CUtensorMap tmWh, const __grid_constant__ CUtensorMap tmWl,
@@ -293,7 +297,7 @@ tc32_linear_kernel(const __grid_constant__ CUtensorMap tmXh, const __grid_consta
                                         a[j * 4 + 2] += prev.z; a[j * 4 + 3] += prev.w;
                                     }
                             }
-                            if (last) epilogue32_f32(a, p, bias_t ? bias_t + c * 32 : nullptr, row, n0 + cb + c * 32, row_ok);
+                            if (last) epilogue32_f32<ACT>(a, p, bias_t ? bias_t + c * 32 : nullptr, row, n0 + cb + c * 32, row_ok);
                             if (row_ok) {
 #pragma unroll
                                 for (int j = 0; j < 8; ++j)
@@ -377,7 +381,13 @@ size_t tc32_split_bytes(long long M, long long N, long long K) {
 
 // shapes the 3xTF32 kernel serves: at least two row blocks (CTA pairs) and enough work to pay for the split
 bool tc32_shape_ok(long long M, long long N, long long K) {
-    return M > BM && K >= 32 && K % 4 == 0 && N % 4 == 0 && 2.0 * (double)M * (double)N * (double)K >= 4.0e9;
+    // three launches (two operand splits and the GEMM) cost about 0.03 ms; from about 6e7 flop on they beat the
+    // CUDA-core kernels (300 x 520 x 200: 0.034 vs 0.057 ms; 1024^3: 0.067 vs 0.307 ms)
+    static const double min_flops = [] {                   // KF_TC32_MIN_FLOPS moves the gate (sweeps)
+        const char* e = std::getenv("KF_TC32_MIN_FLOPS");
+        return e ? std::atof(e) : 6.0e7;
+    }();
+    return M > BM && K >= 32 && K % 4 == 0 && N % 4 == 0 && 2.0 * (double)M * (double)N * (double)K >= min_flops;
 }
 
 int tc32_default_grid(long long M, long long N) {
@@ -387,22 +397,34 @@ int tc32_default_grid(long long M, long long N) {
     return (int)((units < slots ? units : slots) * 2);
 }
 
-kf_status launch_tc32_linear(const void* X, long long ldx, const void* W, long long ldw, void* Y, long long ldy,
-                             long long M, long long N, long long K, const EpilogueParams& ep, void* ws,
-                             cudaStream_t st, int* grid_out) {
-    {
+namespace {
+template <int ACT>
+kf_status launch_tc32_instance(const cudaLaunchConfig_t& lc, const CUtensorMap& tmXh, const CUtensorMap& tmXl,
+                               const CUtensorMap& tmWh, const CUtensorMap& tmWl, const Tc32Params& p) {
+    auto kernel = tc32_linear_kernel<ACT>;
+    {   // opt in to the large dynamic shared memory once per device
         static std::mutex mu;
         static bool done[64] = {};
         int dev = 0;
         if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return KF_ERR_CUDA;
         std::lock_guard<std::mutex> lock(mu);
         if (!done[dev]) {
-            if (cudaFuncSetAttribute(tc32_linear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)kSmemAlloc) != cudaSuccess)
+            if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemAlloc) != cudaSuccess)
                 return KF_ERR_CUDA;
             done[dev] = true;
         }
     }
+    if (cudaLaunchKernelEx(&lc, kernel, tmXh, tmXl, tmWh, tmWl, p) != cudaSuccess) {
+        cudaGetLastError();
+        return KF_ERR_CUDA;
+    }
+    return KF_OK;
+}
+}  // namespace
+
+kf_status launch_tc32_linear(const void* X, long long ldx, const void* W, long long ldw, void* Y, long long ldy,
+                             long long M, long long N, long long K, const EpilogueParams& ep, void* ws,
+                             cudaStream_t st, int* grid_out) {
     uint8_t* cur = static_cast<uint8_t*>(ws) + kStatusBytes;
     float* Xh = reinterpret_cast<float*>(cur); cur += round256((size_t)M * K * 4);
     float* Xl = reinterpret_cast<float*>(cur); cur += round256((size_t)M * K * 4);
@@ -452,11 +474,15 @@ kf_status launch_tc32_linear(const void* X, long long ldx, const void* W, long l
     at[0].val.clusterDim.z = 1;
     lc.attrs = at;
     lc.numAttrs = 1;
-    if (cudaLaunchKernelEx(&lc, tc32_linear_kernel, tmXh, tmXl, tmWh, tmWl, p) != cudaSuccess) {
-        cudaGetLastError();
-        return KF_ERR_CUDA;
+    switch (ep.act) {
+    case KF_ACT_NONE: return launch_tc32_instance<KF_ACT_NONE>(lc, tmXh, tmXl, tmWh, tmWl, p);
+    case KF_ACT_GELU_ERF: return launch_tc32_instance<KF_ACT_GELU_ERF>(lc, tmXh, tmXl, tmWh, tmWl, p);
+    case KF_ACT_GELU_TANH: return launch_tc32_instance<KF_ACT_GELU_TANH>(lc, tmXh, tmXl, tmWh, tmWl, p);
+    case KF_ACT_SILU: return launch_tc32_instance<KF_ACT_SILU>(lc, tmXh, tmXl, tmWh, tmWl, p);
+    case KF_ACT_RELU: return launch_tc32_instance<KF_ACT_RELU>(lc, tmXh, tmXl, tmWh, tmWl, p);
+    case KF_ACT_SIGMOID: return launch_tc32_instance<KF_ACT_SIGMOID>(lc, tmXh, tmXl, tmWh, tmWl, p);
+    default: return KF_ERR_INVALID_ARG;
     }
-    return KF_OK;
 }
 
 }  // namespace kf

@@ -329,6 +329,18 @@ def test_tc32_matches_oracle_under_the_fp32_gate(kf, norm):
     assert r["max_abs"] < 2e-5
 
 
+@pytest.mark.parametrize("act", ACTS)
+def test_tc32_small_shapes_every_activation(kf, act):
+    """fp32 calls from about 6e7 flop on take the tensor cores (three TF32 passes): small ragged shapes, every
+    activation in its accurate form (one kernel instantiation each), with and without a row-norm."""
+    i = ACTS.index(act)
+    M, N, K = [(300, 520, 200), (130, 1028, 260), (515, 520, 132)][i % 3]
+    norm = ["none", "softmax", "layernorm", "rmsnorm"][i % 4]
+    p = make("f32", M, N, K, seed=95 + i, act=act, norm=norm, res=i % 2 == 0, scale=[1.0, 0.5][i % 2])
+    assert kf.tile_config(M, N, K, torch.float32, norm)["kernel"] == 4
+    assert_parity(run(kf, p), oracle_of(p), "f32", f"tc32 {act} {norm} {M}x{N}x{K}")
+
+
 def test_calls_on_a_side_stream_and_growing_workspace(kf):
     """The library launches on the stream it is given: results computed on a side stream, with the
     binding's cached workspace growing between calls of different sizes, match the oracle."""
