@@ -30,7 +30,7 @@
  *   - Alignment: fast paths need 16-byte aligned base pointers and row pitches; anything else
  *     is served by slower generic kernels, never by the CPU.  There is no CPU fallback.
  *   - fp32 calls never take a single TF32 pass (10 mantissa bits miss the 1e-4 gate): small or
- *     unaligned ones run on CUDA cores, large aligned ones (M > 128, 2MNK >= 4e9) on the tensor
+ *     unaligned ones run on CUDA cores, aligned ones from 2MNK >= 6e7 on run on the tensor
  *     cores through three error-compensated TF32 passes with K accumulated in fp32-summed chunks;
  *     those need ws room for hi / lo copies of X and W (kf_workspace_bytes accounts for it).
  *   - M == 0 or N == 0: returns KF_OK and writes nothing.  K == 0: the accumulator is 0.

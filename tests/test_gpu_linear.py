@@ -334,7 +334,7 @@ def test_tc32_small_shapes_every_activation(kf, act):
     """fp32 calls from about 6e7 flop on take the tensor cores (three TF32 passes): small ragged shapes, every
     activation in its accurate form (one kernel instantiation each), with and without a row-norm."""
     i = ACTS.index(act)
-    M, N, K = [(300, 520, 200), (130, 1028, 260), (515, 520, 132)][i % 3]
+    M, N, K = [(300, 520, 200), (130, 1028, 260), (515, 520, 132), (100, 1028, 516), (7, 2056, 4100)][i % 5]
     norm = ["none", "softmax", "layernorm", "rmsnorm"][i % 4]
     p = make("f32", M, N, K, seed=95 + i, act=act, norm=norm, res=i % 2 == 0, scale=[1.0, 0.5][i % 2])
     assert kf.tile_config(M, N, K, torch.float32, norm)["kernel"] == 4
