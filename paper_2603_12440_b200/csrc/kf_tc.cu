@@ -259,18 +259,48 @@ size_t tc_partials_bytes(long long M, long long N) {
     return (size_t)tm * BM * nsub * sizeof(float4);
 }
 
-// K slices per tile for a single row block with a long K: when the tiles alone leave most SMs idle, a cluster of
-// 2, 4 or 8 CTAs shares each tile's K range, as many as still fit the device.  The exchange costs two
-// cluster barriers and a second cold pass through the epilogue code, which a K below ~6000 does not
-// pay back (measured: 64 x 4096 x 4096 the same with and without, 128 x 2048 x 8192 0.059 -> 0.027 ms).
+// clusters of c single CTAs of the GEMM kernel that the device holds at once: a cluster lives inside one GPC, so
+// this is below SMs / c (B200: 16 clusters of 8 do not fit although 128 <= 148).  Asked of the runtime once per
+// size; without a device (host-only callers of the tile table) the figures of a B200 are assumed.
+static int tc_max_clusters(int c) {
+    static std::mutex mu;
+    static int cached[9] = {};
+    std::lock_guard<std::mutex> lock(mu);
+    if (cached[c]) return cached[c];
+    int fallback = c == 8 ? 8 : (c == 4 ? 32 : 64), n = 0, dev = 0;
+    auto kernel = tc_linear_kernel<1, -1, -1>;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemAlloc) == cudaSuccess) {
+        cudaLaunchConfig_t lc = {};
+        lc.gridDim = dim3((unsigned)(c * 64));
+        lc.blockDim = dim3(kThreads);
+        lc.dynamicSmemBytes = kSmemAlloc;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = (unsigned)c;
+        at[0].val.clusterDim.y = 1;
+        at[0].val.clusterDim.z = 1;
+        lc.attrs = at;
+        lc.numAttrs = 1;
+        if (cudaOccupancyMaxActiveClusters(&n, kernel, &lc) != cudaSuccess || n <= 0) n = 0;
+    }
+    cudaGetLastError();
+    cached[c] = n > 0 ? n : fallback;
+    return cached[c];
+}
+
+// K slices per tile for a single row block: when the tiles alone leave most SMs idle, a cluster of 2, 4 or 8
+// CTAs shares each tile's K range -- the most slices that keep every cluster resident at once and leave each
+// slice at least 16 k-blocks (below that the exchange, two cluster barriers and a second pass through the
+// epilogue code, costs more than the shorter main loop saves).  Measured: 64 x 4096 x 4096 0.037 -> 0.025 ms
+// with 4 slices, 128 x 8192 x 2048 0.027 -> 0.023 with 2 (0.025 with 4), 128 x 2048 x 8192 0.059 -> 0.027 with 8.
 int tc_default_splitk(long long M, long long N, long long K, int cta_group) {
     if (cta_group != 1 || M > BM) return 1;
     const long long tiles = (N + BN - 1) / BN, kblocks = (K + BK - 1) / BK;
-    if (kblocks < 96) return 1;
     int sk = 1;
     for (int c = 2; c <= 8; c *= 2) {
         const long long per = (kblocks + c - 1) / c;       // k-blocks per slice: every slice must get at least one
-        if (tiles * c <= sm_count() && kblocks >= 2 * c && (c - 1) * per < kblocks) sk = c;
+        if (tiles <= tc_max_clusters(c) && per >= 16 && (c - 1) * per < kblocks) sk = c;
     }
     return sk;
 }
@@ -331,7 +361,7 @@ kf_status launch_tc_linear(const void* X, long long ldx, const void* W, long lon
     if (env_sk == 1) p.splitk = 1;
     if ((env_sk == 2 || env_sk == 4 || env_sk == 8) && cta_group == 1 && M <= BM) {     // forced where the slices are legal
         const long long tiles = (N + BN - 1) / BN, kblocks = (K + BK - 1) / BK, per = (kblocks + env_sk - 1) / env_sk;
-        if (tiles * env_sk <= sm_count() && kblocks >= 2 * env_sk && (env_sk - 1) * per < kblocks) p.splitk = env_sk;
+        if (tiles <= tc_max_clusters(env_sk) && kblocks >= 2 * env_sk && (env_sk - 1) * per < kblocks) p.splitk = env_sk;
     }
     int grid = tc_default_grid(M, N, cta_group);
     if (p.splitk > 1) {
