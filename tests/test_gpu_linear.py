@@ -172,9 +172,11 @@ def test_tc_tall_and_very_wide_rownorm(kf, M, N, K, norm):
 
 @pytest.mark.parametrize("M,N,K,norm", [(128, 2056, 8200, "layernorm"),      # 9 tiles x 8 K slices
                                          (70, 9480, 6160, "softmax"),          # 38 tiles x 2 slices, ragged everywhere
-                                         (1, 520, 12296, "none")])             # 3 tiles x 8 slices, one row
+                                         (1, 520, 12296, "none"),              # 3 tiles x 8 slices, one row
+                                         (100, 264, 2056, "rmsnorm"),          # 33 k-blocks: 2 slices of 17 and 16
+                                         (90, 1032, 4104, "none")])            # 65 k-blocks: 4 slices, the last of 14
 def test_tc_split_k_single_row_block(kf, M, N, K, norm):
-    """One row block and a long K: the K range of a tile is shared by the CTAs of a cluster and the partial
+    """One row block: the K range of a tile is shared by the CTAs of a cluster and the partial
     accumulators are added in the owner's shared memory before the epilogue."""
     p = make("bf16", M, N, K, seed=71 + M, act="gelu_erf", norm=norm, res=True)
     assert kf.tile_config(M, N, K, torch.bfloat16, norm)["cta_group"] == 1
