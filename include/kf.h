@@ -97,13 +97,15 @@ typedef struct {
 /* Which kernel and tile shape a call resolves to (the hardware-aware table, Section 3.4:
  * the best-measured instantiation of a templated kernel is the one that is used). */
 typedef struct {
-    int32_t kernel;           /* 0 none, 1 SIMT row-resident, 2 SIMT tiled, 3 tcgen05 bf16, 4 tcgen05 fp32 (3xTF32) */
+    int32_t kernel;           /* 0 none, 1 SIMT row-resident, 2 SIMT tiled, 3 tcgen05 bf16, 4 tcgen05 fp32 (3xTF32),
+                                 5 SIMT rows dealt over a cluster (small fp32) */
     int32_t bm, bn, bk;       /* tile of one work unit (a CTA, or a CTA pair when cta_group is 2) */
     int32_t stages;           /* shared-memory pipeline depth */
     int32_t cta_group;        /* 1 or 2 CTAs per MMA */
     int32_t epilogue_warps;
     int32_t row_scheme;       /* 0 none, 1 in-CTA rows, 2 split-N partials + normalise pass,
-                                 3 split-N partials + in-kernel deferred normalise, 4 un-fused */
+                                 3 split-N partials + in-kernel deferred normalise, 4 un-fused,
+                                 5 row dealt over a cluster, statistics through distributed shared memory */
     int32_t grid;             /* CTAs launched by the main kernel */
 } kf_tile_config;
 

@@ -33,7 +33,7 @@ const Override& env_override() {
 }
 
 // The table.  Shape classes and their winners; tensor-core rows carry the tile the kernel was
-// built with.  kernel: 1 SIMT row-resident, 2 SIMT tiled, 3 tcgen05.
+// built with.  kernel: 1 SIMT row-resident, 2 SIMT tiled, 3 tcgen05, 4 tcgen05 3xTF32, 5 SIMT rows over a cluster.
 kf_status resolve(long long M, long long N, long long K, int dt, int norm, bool aligned, kf_tile_config* c) {
     std::memset(c, 0, sizeof(*c));
     if (M == 0 || N == 0) return KF_OK;
@@ -60,6 +60,15 @@ kf_status resolve(long long M, long long N, long long K, int dt, int norm, bool 
         c->bm = 256; c->bn = 256; c->bk = 32; c->stages = 3; c->cta_group = 2; c->epilogue_warps = 8;
         c->row_scheme = norm == KF_NORM_NONE ? 0 : 4;
         c->grid = tc32_default_grid(M, N);
+        return KF_OK;
+    }
+    // small aligned fp32 with a short row: latency-bound, a cluster of 8 CTAs shares each group of 8 rows
+    if (dt == KF_F32 && aligned && simt_cluster_ok(M, N, K) && ov.kernel != 1 && ov.kernel != 2) {
+        c->kernel = 5;
+        c->bm = 8; c->bn = (int)N; c->bk = (N + 7) / 8 <= 32 ? 256 : 128; c->stages = 1; c->cta_group = 1;
+        c->epilogue_warps = 8;
+        c->row_scheme = norm == KF_NORM_NONE ? 0 : 5;
+        c->grid = (int)(((M + 7) / 8) * 8);
         return KF_OK;
     }
     bool rows = simt_row_resident_ok(N) && (norm != KF_NORM_NONE ? (M < 4096 || dt == KF_BF16) : (M <= 1024));
@@ -142,6 +151,8 @@ kf_status linear_impl(const void* X, int64_t ldx, const void* W, int64_t ldw, vo
         if (s != KF_OK || rn.norm == KF_NORM_NONE) return s;
         return launch_row_norm(Y, ldy, Y, ldy, M, N, dt, rn, st) == cudaSuccess ? KF_OK : KF_ERR_CUDA;
     }
+    if (cfg.kernel == 5)
+        return launch_simt_cluster(X, ldx, W, ldw, Y, ldy, M, N, K, ep, rn, st, nullptr) == cudaSuccess ? KF_OK : KF_ERR_CUDA;
     cudaError_t e = launch_simt_linear(X, ldx, W, ldw, Y, ldy, M, N, K, dt, ep, rn, cfg.kernel == 1, st, nullptr);
     return e == cudaSuccess ? KF_OK : KF_ERR_CUDA;
 }

@@ -153,5 +153,10 @@ cudaError_t launch_simt_linear(const void* X, long long ldx, const void* W, long
                                const EpilogueParams& ep, const RowNormParams& rn, bool row_resident,
                                cudaStream_t st, int* grid_out);
 bool simt_row_resident_ok(long long N);
+// small fp32 calls: the columns of 8 rows dealt over a cluster of 8 CTAs (kf_simt_cluster.cu)
+bool simt_cluster_ok(long long M, long long N, long long K);
+cudaError_t launch_simt_cluster(const void* X, long long ldx, const void* W, long long ldw, void* Y, long long ldy,
+                                long long M, long long N, long long K, const EpilogueParams& ep,
+                                const RowNormParams& rn, cudaStream_t st, int* grid_out);
 
 }  // namespace kf

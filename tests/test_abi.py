@@ -54,7 +54,10 @@ def test_workspace_bytes(kf):
 def test_tile_table_on_the_five_configs(kf):
     import torch
     c1 = kf.tile_config(128, 256, 256, torch.float32, "softmax")
-    assert c1["kernel"] == 1 and c1["row_scheme"] == 1            # fp32: CUDA cores, rows resident in a CTA
+    # small fp32: CUDA cores, each group of 8 rows dealt over a cluster of 8 CTAs (16 clusters)
+    assert (c1["kernel"], c1["row_scheme"], c1["bm"], c1["grid"]) == (5, 5, 8, 128)
+    long_rows = kf.tile_config(128, 1024, 128, torch.float32, "softmax")     # rows resident in a CTA
+    assert long_rows["kernel"] == 1 and long_rows["row_scheme"] == 1
     c3 = kf.tile_config(8192, 4096, 4096, torch.bfloat16, "none")
     # large bf16: CTA pairs (cta_group 2) computing 256 x 256 per work unit from a 6-stage ring
     assert (c3["kernel"], c3["bm"], c3["bn"], c3["bk"], c3["cta_group"], c3["stages"], c3["row_scheme"]) == \

@@ -47,7 +47,7 @@ def make(dtype, M, N, K, seed, act="none", norm="none", bias=True, res=False, sc
 # ------------------------------------------------------------------------------- fp32 (CUDA cores)
 def test_config1_fp32_full(kf):
     p = inputs.config(1)
-    assert kf.tile_config(p.M, p.N, p.K, torch.float32, p.norm)["kernel"] == 1
+    assert kf.tile_config(p.M, p.N, p.K, torch.float32, p.norm)["kernel"] == 5     # rows dealt over clusters
     r = assert_parity(run(kf, p), oracle_of(p), "f32", "C1")
     assert r["max_abs"] < 1e-6                      # far inside the 1e-4 gate
     # the pre-norm values through kf_linear_epilogue (values ~0.06) under the same 1e-4 gate
@@ -62,12 +62,32 @@ def test_fp32_activations_row_resident(kf, act):
 
 
 @pytest.mark.parametrize("norm", ["softmax", "layernorm", "rmsnorm"])
-@pytest.mark.parametrize("M,N,K", [(1, 1, 1), (5, 7, 3), (33, 256, 64), (300, 257, 100), (17, 1000, 77), (9, 2048, 40),
-                                   (3, 40, 0)])
+@pytest.mark.parametrize("M,N,K", [(1, 1, 1), (5, 7, 3), (33, 256, 66), (300, 257, 100), (17, 1000, 77), (9, 2048, 40),
+                                   (3, 40, 0), (2100, 256, 8)])
 def test_fp32_rownorm_row_resident(kf, norm, M, N, K):
     p = make("f32", M, N, K, seed=12 + N, act="gelu_erf", norm=norm, res=True)
-    assert kf.tile_config(M, N, K, torch.float32, norm)["kernel"] == 1
+    aligned = N % 4 == 0 and K % 4 == 0                  # row pitches of the contiguous test tensors
+    assert kf.tile_config(M, N, K, torch.float32, norm, aligned=aligned)["kernel"] == 1
     assert_parity(run(kf, p), oracle_of(p), "f32", f"{norm} {M}x{N}x{K}")
+
+
+@pytest.mark.parametrize("norm", ["none", "softmax", "layernorm", "rmsnorm"])
+@pytest.mark.parametrize("M,N,K", [(33, 256, 64),        # one slab, 32 columns per CTA
+                                   (1, 64, 256),         # one row, 8 columns per CTA
+                                   (100, 200, 260),      # 25 columns per CTA, a second slab of 4
+                                   (9, 264, 516),        # 33 columns per CTA: two per lane, five slabs of 128
+                                   (77, 68, 1028),       # 9 columns per CTA, the last CTA has 5
+                                   (256, 512, 32)])      # the most rows and the longest row this kernel takes
+def test_fp32_small_calls_rows_over_a_cluster(kf, norm, M, N, K):
+    """Small aligned fp32 calls: 8 rows per cluster of 8 CTAs, each CTA an eighth of the columns, the row
+    statistics merged through distributed shared memory."""
+    i = (M + N + K) % 6
+    p = make("f32", M, N, K, seed=15 + N, act=ACTS[i], norm=norm, res=i % 2 == 0, scale=[1.0, 0.5][i % 2])
+    cfg = kf.tile_config(M, N, K, torch.float32, norm)
+    assert cfg["kernel"] == 5 and cfg["grid"] == (M + 7) // 8 * 8 and cfg["row_scheme"] == (0 if norm == "none" else 5)
+    got = run(kf, p)
+    assert_parity(got, oracle_of(p), "f32", f"cluster {norm} {M}x{N}x{K}")
+    assert np.array_equal(got, run(kf, p))                  # fixed summation order
 
 
 @pytest.mark.parametrize("norm", ["none", "softmax", "layernorm"])
