@@ -7,10 +7,11 @@
 //   one round trip); warp w then multiplies the w-th eighth of the slab's k range for all 8 rows, lane =
 //   column, so each W value leaves shared memory once; the eight partial sums of an output are added in
 //   a fixed order through shared memory, after which warp = row, lane = column.
-//   row statistics: each CTA reduces its slice of the 8 rows (one warp per row), pushes one float2 per row
-//   into every CTA of the cluster through distributed shared memory, and merges the eight pairs after a
-//   single cluster barrier: softmax (max, sum of exp about it), LayerNorm (mean, sum of squared
-//   deviations; Chan's merge), RMSNorm (sum of squares).
+//   row statistics: each CTA reduces its slice of the 8 rows (one warp per row) to one float2 per row in its
+//   own shared memory -- softmax (max, sum of exp about it), LayerNorm (mean, sum of squared deviations;
+//   Chan's merge), RMSNorm (sum of squares) -- and after one cluster barrier reads the other seven CTAs'
+//   pairs through distributed shared memory; a second barrier, whose wait is the last thing a CTA does,
+//   keeps every CTA's shared memory alive until all have read it.
 #include <cooperative_groups.h>
 
 #include "kf_common.cuh"
@@ -40,7 +41,7 @@ simt_cluster_kernel(const float* __restrict__ X, long long ldx, const float* __r
     static_assert(NCOLS * PQ >= 8 * kRowsCl * NCOLS / 4, "the partial sums reuse the W slab");
     __shared__ float4 ws4[NCOLS * PQ];
     __shared__ float4 xs4[kRowsCl * KQ];
-    __shared__ float2 exch[kRowsCl][kCl];
+    __shared__ float2 exch[kRowsCl];
 
     cg::cluster_group cluster = cg::this_cluster();
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
@@ -49,10 +50,6 @@ simt_cluster_kernel(const float* __restrict__ X, long long ldx, const float* __r
     const int NC = (N + kCl - 1) / kCl;
     const int n_base = rank * NC;
     const int ncols = max(0, min(NC, N - n_base));           // columns this CTA really has
-    // every CTA of the cluster must be running before its shared memory is written from outside:
-    // arrive now, wait just before the exchange
-    if (norm != KF_NORM_NONE) cluster.barrier_arrive();
-
     float4 wreg[WU], xreg[XU];
     auto load_slab = [&](int k0) {
 #pragma unroll
@@ -170,12 +167,16 @@ simt_cluster_kernel(const float* __restrict__ X, long long ldx, const float* __r
             for (int j = 0; j < CPL; ++j) q = fmaf(a[j], a[j], q);           // a is 0 where there is no column
             mine = make_float2(0.f, warp_sum(q));
         }
-        cluster.barrier_wait();                              // (the arrive at the top) every CTA is running
-        if (lane < kCl) *cluster.map_shared_rank(&exch[warp][rank], lane) = mine;
-        cluster.sync();                                      // release the pushes, acquire the others'
+        // every CTA publishes its pairs in its own shared memory; after the barrier (which also says that every
+        // CTA of the cluster is running) lane p reads CTA p's pair of this row, and the warp shares them out
+        if (lane == 0) exch[warp] = mine;
+        cluster.sync();
+        const float2 theirs = lane < kCl ? *cluster.map_shared_rank(&exch[warp], lane) : make_float2(0.f, 0.f);
+        cluster.barrier_arrive();                            // this CTA has read; waited for before it exits
         float2 part[kCl];
 #pragma unroll
-        for (int p = 0; p < kCl; ++p) part[p] = exch[warp][p];
+        for (int p = 0; p < kCl; ++p)
+            part[p] = make_float2(__shfl_sync(0xFFFFFFFFu, theirs.x, p), __shfl_sync(0xFFFFFFFFu, theirs.y, p));
         if (norm == KF_NORM_SOFTMAX) {
             float m = part[0].x;                             // CTA 0 always has a column
 #pragma unroll
@@ -213,6 +214,7 @@ simt_cluster_kernel(const float* __restrict__ X, long long ldx, const float* __r
 #pragma unroll
     for (int j = 0; j < CPL; ++j)
         if (ok[j]) Y[(long long)row * ldy + n_base + lane + 32 * j] = a[j];
+    if (norm != KF_NORM_NONE) cluster.barrier_wait();        // no CTA leaves while another may still read its pairs
 }
 
 template <int CPL>
