@@ -6,6 +6,8 @@
 // LayerNorm takes both moments in one sweep about a shift from the row itself (one reduction round).
 // Generic path (row length or pointers not 16-byte friendly, or rows too long for registers):
 // one CTA per row, scalar accesses, three passes over global memory.
+#include <cuda_fp16.h>
+
 #include "kf_common.cuh"
 
 #include <cstdlib>
@@ -20,6 +22,32 @@ constexpr int kRowThreads = 256;
 // instruction count to show (long LayerNorm rows most of all).
 __device__ __forceinline__ float2 pr2(const float* f, int k) { return make_float2(f[2 * k], f[2 * k + 1]); }
 __device__ __forceinline__ float2 dup2(float x) { return make_float2(x, x); }
+
+// The softmax kernels take exp once per element: between the sum sweep and the output sweep the values
+// e = exp(x - max) in (0, 1] stay in the 16 bytes their inputs came in -- fp32 as they are, 16-bit inputs as
+// fp16 (11 significant bits, four times finer than the bf16 the result is rounded to; below 2^-24 they
+// flush to 0, far under what a bf16 softmax output can show).  The sum is taken from the fp32 values.
+template <typename T> __device__ __forceinline__ uint4 pack_e(const float* f);
+template <> __device__ __forceinline__ uint4 pack_e<float>(const float* f) { return pack<float>(f); }
+template <> __device__ __forceinline__ uint4 pack_e<__nv_bfloat16>(const float* f) {
+    uint4 r;
+    __half2 h;
+    h = __floats2half2_rn(f[0], f[1]); r.x = *reinterpret_cast<uint32_t*>(&h);
+    h = __floats2half2_rn(f[2], f[3]); r.y = *reinterpret_cast<uint32_t*>(&h);
+    h = __floats2half2_rn(f[4], f[5]); r.z = *reinterpret_cast<uint32_t*>(&h);
+    h = __floats2half2_rn(f[6], f[7]); r.w = *reinterpret_cast<uint32_t*>(&h);
+    return r;
+}
+template <typename T> __device__ __forceinline__ void unpack_e(const uint4& v, float* f);
+template <> __device__ __forceinline__ void unpack_e<float>(const uint4& v, float* f) { unpack<float>(v, f); }
+template <> __device__ __forceinline__ void unpack_e<__nv_bfloat16>(const uint4& v, float* f) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const float2 p = __half22float2(*reinterpret_cast<const __half2*>(&w[k]));
+        f[2 * k] = p.x; f[2 * k + 1] = p.y;
+    }
+}
 
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) { return __ldcs(p); }
 __device__ __forceinline__ void st_stream(uint4* p, const uint4& v) { __stcs(p, v); }
@@ -96,8 +124,11 @@ row_norm_reg_kernel(const T* X, long long ldx, T* Y, long long ldy, long long M,
 #pragma unroll
                 for (int k = 0; k < E / 2; ++k) {
                     const float2 t = __ffma2_rn(pr2(f, k), l2e, nms);
-                    s2 = __fadd2_rn(s2, make_float2(fast_ex2(t.x), fast_ex2(t.y)));
+                    const float2 e2 = make_float2(fast_ex2(t.x), fast_ex2(t.y));
+                    s2 = __fadd2_rn(s2, e2);
+                    f[2 * k] = e2.x; f[2 * k + 1] = e2.y;
                 }
+                v[i] = pack_e<T>(f);                         // the exp values take the place of their inputs
             }
         const float s = group_reduce<false>(s2.x + s2.y, tpr, red);
         const float2 inv = dup2(1.0f / s);
@@ -105,11 +136,10 @@ row_norm_reg_kernel(const T* X, long long ldx, T* Y, long long ldy, long long M,
         for (int i = 0; i < VPT; ++i) {
             const int idx = lr + i * tpr;
             if (live && idx < NV) {
-                unpack<T>(v[i], f);
+                unpack_e<T>(v[i], f);
 #pragma unroll
                 for (int k = 0; k < E / 2; ++k) {
-                    const float2 t = __ffma2_rn(pr2(f, k), l2e, nms);
-                    const float2 o = __fmul2_rn(make_float2(fast_ex2(t.x), fast_ex2(t.y)), inv);
+                    const float2 o = __fmul2_rn(pr2(f, k), inv);
                     f[2 * k] = o.x; f[2 * k + 1] = o.y;
                 }
                 st_stream(yr + idx, pack<T>(f));
@@ -328,19 +358,22 @@ row_norm_ring_kernel(const T* X, long long ldx, T* Y, long long ldy, long long M
 #pragma unroll
                     for (int k = 0; k < E / 2; ++k) {
                         const float2 t = __ffma2_rn(pr2(x, k), l2e, nms);
-                        l[k & 1] = __fadd2_rn(l[k & 1], make_float2(fast_ex2(t.x), fast_ex2(t.y)));
+                        const float2 e2 = make_float2(fast_ex2(t.x), fast_ex2(t.y));
+                        l[k & 1] = __fadd2_rn(l[k & 1], e2);
+                        x[2 * k] = e2.x; x[2 * k + 1] = e2.y;
                     }
+                    // the exp values take the place of their inputs in the slot (each lane its own vectors)
+                    const_cast<uint4*>(srow)[lane + v * 32] = pack_e<T>(x);
                 }
             const float2 inv = dup2(1.0f / warp_sum((l[0].x + l[0].y) + (l[1].x + l[1].y)));
 #pragma unroll
             for (int v = 0; v < VPT; ++v) {
                 const int idx = lane + v * 32;
                 if (idx < NV) {
-                    unpack<T>(srow[idx], x);
+                    unpack_e<T>(srow[idx], x);
 #pragma unroll
                     for (int k = 0; k < E / 2; ++k) {
-                        const float2 t = __ffma2_rn(pr2(x, k), l2e, nms);
-                        const float2 o = __fmul2_rn(make_float2(fast_ex2(t.x), fast_ex2(t.y)), inv);
+                        const float2 o = __fmul2_rn(pr2(x, k), inv);
                         x[2 * k] = o.x; x[2 * k + 1] = o.y;
                     }
                     st_stream(yr + idx, pack<T>(x));
@@ -391,8 +424,10 @@ row_norm_ring_kernel(const T* X, long long ldx, T* Y, long long ldy, long long M
             }
         }
         }                                                   // rows of the block
+        // softmax wrote its exp values into the slot: order those writes before the bulk copy that refills it
+        if (NORM == KF_NORM_SOFTMAX) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
-        if (lane == 0) rbar_arrive(empty_bar(s));           // every lane has finished reading the slot
+        if (lane == 0) rbar_arrive(empty_bar(s));           // every lane has finished with the slot
     }
 }
 
