@@ -431,6 +431,181 @@ row_norm_ring_kernel(const T* X, long long ldx, T* Y, long long ldy, long long M
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Group ring: the ring kernel for rows of 8 to 64 KiB.  A slot holds one row and a group of G consumer
+// warps (16 / G groups) shares it: lane-strided over the row's vectors, statistics reduced inside the
+// warp and then across the group through shared memory and a named barrier of the group's threads.
+// gamma / beta stay in the input type (a row's worth of shared memory each); a slot always returns to
+// the same group (slots are a multiple of the groups).  A wait that gives up raises the group's abort
+// flag; the group reads it after its next barrier and leaves together, so no warp is left at a barrier.
+constexpr int kGringWarps = 16;
+
+template <typename T, int NORM, int G>
+__global__ void __launch_bounds__(32 * (kGringWarps + 1), 1)
+row_norm_gring_kernel(const T* X, long long ldx, T* Y, long long ldy, long long M, int N, int slots,   // Y may be X
+                      const T* __restrict__ gamma, const T* __restrict__ beta, float eps) {
+    constexpr int E = Elem<T>::kVec;
+    constexpr int NG = kGringWarps / G, GT = 32 * G;
+    extern __shared__ __align__(128) uint8_t ring_smem[];
+    const int NV = N / E;
+    const uint32_t row_bytes = (uint32_t)N * sizeof(T);
+    // layout: [slots x row][gamma row][beta row][reductions][abort flags][barriers]
+    uint8_t* ring = ring_smem;
+    uint4* gam = reinterpret_cast<uint4*>(ring_smem + (size_t)slots * row_bytes);
+    uint4* bet = gam + (NORM == KF_NORM_SOFTMAX ? 0 : NV);
+    float2* redA = reinterpret_cast<float2*>(bet + (NORM == KF_NORM_LAYERNORM ? NV : 0));    // [2][16]
+    float2* redB = redA + 2 * kGringWarps;                                                   // [2][16]
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(redB + 2 * kGringWarps);      // [8]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(const_cast<int*>(abort_flag) + 8);
+    const uint32_t bar0 = smem_addr(bars);
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (slots + s); };
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < slots; ++s) {
+            rbar_init(full_bar(s), 1);
+            rbar_init(empty_bar(s), G);
+        }
+        for (int g = 0; g < 8; ++g) abort_flag[g] = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    const long long my_rows = (M - blockIdx.x + gridDim.x - 1) / gridDim.x;      // rows blockIdx.x, + gridDim.x, ...
+
+    if (warp == kGringWarps) {
+        if (lane == 0) {
+            for (long long i = 0; i < my_rows; ++i) {
+                const int s = (int)(i % slots);
+                const uint32_t ph = (uint32_t)((i / slots) & 1);
+                if (!rbar_wait(empty_bar(s), ph ^ 1u)) break;
+                const long long row = blockIdx.x + i * (long long)gridDim.x;
+                rbar_expect_tx(full_bar(s), row_bytes);
+                bulk_load_row(smem_addr(ring + (size_t)s * row_bytes), X + row * ldx, row_bytes, full_bar(s));
+            }
+        }
+        return;
+    }
+
+    if (NORM != KF_NORM_SOFTMAX) {
+        float one[E], zero[E];
+#pragma unroll
+        for (int e = 0; e < E; ++e) { one[e] = 1.f; zero[e] = 0.f; }
+        for (int idx = threadIdx.x; idx < NV; idx += kGringWarps * 32) {
+            gam[idx] = gamma ? __ldg(reinterpret_cast<const uint4*>(gamma) + idx) : pack<T>(one);
+            if (NORM == KF_NORM_LAYERNORM) bet[idx] = beta ? __ldg(reinterpret_cast<const uint4*>(beta) + idx) : pack<T>(zero);
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(kGringWarps * 32) : "memory");
+    }
+
+    const int g = warp / G, gl = (warp % G) * 32 + lane, w0 = g * G;
+    auto group_bar = [&]() { asm volatile("bar.sync %0, %1;" ::"r"(2 + g), "n"(GT) : "memory"); };
+    for (long long i = g; i < my_rows; i += NG) {
+        const int s = (int)(i % slots);
+        const uint32_t ph = (uint32_t)((i / slots) & 1);
+        const int par = (int)((i / NG) & 1);                 // the reduction buffers alternate from row to row
+        const long long row = blockIdx.x + i * (long long)gridDim.x;
+        if (!rbar_wait(full_bar(s), ph)) abort_flag[g] = 1;
+        uint4* srow = reinterpret_cast<uint4*>(ring + (size_t)s * row_bytes);
+        uint4* yr = reinterpret_cast<uint4*>(Y + row * ldy);
+        float x[E];
+        if (NORM == KF_NORM_SOFTMAX) {
+            float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll 4
+            for (int idx = gl; idx < NV; idx += GT) {
+                unpack<T>(srow[idx], x);
+#pragma unroll
+                for (int e = 0; e < E; ++e) m4[e & 3] = fmaxf(m4[e & 3], x[e]);
+            }
+            const float mw = warp_max(fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])));
+            if (lane == 0) redA[par * kGringWarps + warp].x = mw;
+            group_bar();
+            if (abort_flag[g]) break;
+            float m = redA[par * kGringWarps + w0].x;
+#pragma unroll
+            for (int w = 1; w < G; ++w) m = fmaxf(m, redA[par * kGringWarps + w0 + w].x);
+            const float2 l2e = dup2(kLog2e), nms = dup2(-m * kLog2e);
+            float2 l[2] = {dup2(0.f), dup2(0.f)};
+#pragma unroll 4
+            for (int idx = gl; idx < NV; idx += GT) {
+                unpack<T>(srow[idx], x);
+#pragma unroll
+                for (int k = 0; k < E / 2; ++k) {
+                    const float2 t = __ffma2_rn(pr2(x, k), l2e, nms);
+                    const float2 e2 = make_float2(fast_ex2(t.x), fast_ex2(t.y));
+                    l[k & 1] = __fadd2_rn(l[k & 1], e2);
+                    x[2 * k] = e2.x; x[2 * k + 1] = e2.y;
+                }
+                srow[idx] = pack_e<T>(x);                    // exp once: the values take their inputs' place
+            }
+            const float lw = warp_sum((l[0].x + l[0].y) + (l[1].x + l[1].y));
+            if (lane == 0) redB[par * kGringWarps + warp].x = lw;
+            group_bar();
+            float sum = redB[par * kGringWarps + w0].x;
+#pragma unroll
+            for (int w = 1; w < G; ++w) sum += redB[par * kGringWarps + w0 + w].x;
+            const float2 inv = dup2(1.0f / sum);
+#pragma unroll 4
+            for (int idx = gl; idx < NV; idx += GT) {
+                unpack_e<T>(srow[idx], x);
+#pragma unroll
+                for (int k = 0; k < E / 2; ++k) {
+                    const float2 o = __fmul2_rn(pr2(x, k), inv);
+                    x[2 * k] = o.x; x[2 * k + 1] = o.y;
+                }
+                st_stream(yr + idx, pack<T>(x));
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // slot writes before the refill
+        } else {
+            // both moments in one sweep about a shift from the row itself (its first element); RMSNorm: 0
+            const float c = (NORM == KF_NORM_LAYERNORM) ? Elem<T>::load(reinterpret_cast<const T*>(srow)) : 0.f;
+            float2 a[2] = {dup2(0.f), dup2(0.f)}, q[2] = {dup2(0.f), dup2(0.f)};
+            const float2 nc = dup2(-c);
+#pragma unroll 4
+            for (int idx = gl; idx < NV; idx += GT) {
+                unpack<T>(srow[idx], x);
+#pragma unroll
+                for (int k = 0; k < E / 2; ++k) {
+                    const float2 d = __fadd2_rn(pr2(x, k), nc);
+                    a[k & 1] = __fadd2_rn(a[k & 1], d);
+                    q[k & 1] = __ffma2_rn(d, d, q[k & 1]);
+                }
+            }
+            const float s1w = warp_sum((a[0].x + a[0].y) + (a[1].x + a[1].y));
+            const float s2w = warp_sum((q[0].x + q[0].y) + (q[1].x + q[1].y));
+            if (lane == 0) redA[par * kGringWarps + warp] = make_float2(s1w, s2w);
+            group_bar();
+            if (abort_flag[g]) break;
+            float2 t = redA[par * kGringWarps + w0];
+#pragma unroll
+            for (int w = 1; w < G; ++w) {
+                const float2 u = redA[par * kGringWarps + w0 + w];
+                t.x += u.x; t.y += u.y;
+            }
+            const float dm = (NORM == KF_NORM_LAYERNORM) ? t.x / (float)N : 0.f;         // mean - c
+            const float var = fmaxf(t.y / (float)N - dm * dm, 0.f);
+            const float rstd = rsqrtf(var + eps);
+            const float2 rs2 = dup2(rstd), ofs2 = dup2(-(c + dm) * rstd);
+#pragma unroll 4
+            for (int idx = gl; idx < NV; idx += GT) {
+                float gg[E], bb[E];
+                unpack<T>(srow[idx], x);
+                unpack<T>(gam[idx], gg);
+                if (NORM == KF_NORM_LAYERNORM) unpack<T>(bet[idx], bb);
+#pragma unroll
+                for (int k = 0; k < E / 2; ++k) {
+                    float2 o = __fmul2_rn(__ffma2_rn(pr2(x, k), rs2, ofs2), pr2(gg, k));   // (x - mean) rstd gamma
+                    if (NORM == KF_NORM_LAYERNORM) o = __fadd2_rn(o, pr2(bb, k));
+                    x[2 * k] = o.x; x[2 * k + 1] = o.y;
+                }
+                st_stream(yr + idx, pack<T>(x));
+            }
+        }
+        __syncwarp();
+        if (lane == 0) rbar_arrive(empty_bar(s));            // this warp has finished with the slot (G arrivals free it)
+    }
+}
+
 // generic: one CTA per row, scalar accesses, any N / alignment; Y may alias X
 template <typename T, int NORM>
 __global__ void __launch_bounds__(kRowThreads)
@@ -475,6 +650,22 @@ row_norm_generic_kernel(const T* X, long long ldx, T* Y, long long ldy, long lon
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+template <typename T, int NORM, int G>
+cudaError_t launch_gring(const T* x, long long ldx, T* y, long long ldy, long long M, long long N, int slots, int grid,
+                         size_t smem, const T* g, const T* b, float eps, cudaStream_t st) {
+    static bool attr_done[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !attr_done[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(row_norm_gring_kernel<T, NORM, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             226 * 1024);
+        if (e != cudaSuccess) return e;
+        attr_done[dev] = true;
+    }
+    row_norm_gring_kernel<T, NORM, G><<<grid, 32 * (kGringWarps + 1), smem, st>>>(x, ldx, y, ldy, M, (int)N, slots, g, b, eps);
+    return cudaGetLastError();
+}
+
 template <typename T, int NORM>
 cudaError_t launch_typed(const void* X, long long ldx, void* Y, long long ldy, long long M, long long N,
                          const RowNormParams& rn, cudaStream_t st) {
@@ -508,10 +699,11 @@ cudaError_t launch_typed(const void* X, long long ldx, void* Y, long long ldy, l
         if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) return 148;
         return v;
     }();
-    // ring kernel: a row fits one warp's registers, rows start 16-byte aligned, Y does not alias X
-    // (the producer runs ahead of the stores), and there are enough rows to fill persistent CTAs
-    const bool ring_ok = NV <= 32 * 16 && (const void*)X != (const void*)Y && M >= 4ll * sms && env_tpr == 0 &&
-                         env_ring != 0;
+    // ring kernel: a row fits one warp's registers, rows start 16-byte aligned, and there are enough rows to
+    // fill persistent CTAs; in place only as an exact alias (a row is stored after its own copy has landed,
+    // and the copies that run ahead read other rows)
+    const bool ring_ok = NV <= 32 * 16 && ((const void*)X != (const void*)Y || ldx == ldy) && M >= 4ll * sms &&
+                         env_tpr == 0 && env_ring != 0;
     if (ring_ok) {
         const int need_v = (int)((NV + 31) / 32);
         int vpt = 1;
@@ -574,6 +766,29 @@ cudaError_t launch_typed(const void* X, long long ldx, void* Y, long long ldy, l
 #undef KF_RING_LAUNCH
             if (e != cudaSuccess) return e;
             return cudaGetLastError();
+        }
+    }
+    // group ring: rows beyond one warp's reach, up to 64 KiB; in place only as an exact alias.  Not for 16-bit
+    // softmax, where the register kernel already runs at copy speed (8192 / 16384 / 32768-element bf16 rows,
+    // 128 MiB: 0.049 / 0.049 / 0.059 ms there, 0.053 / 0.057 / 0.061 here: two group barriers and three sweeps)
+    const size_t grow_bytes = (size_t)N * sizeof(T);
+    if (NV > 32 * 16 && grow_bytes <= 65536 && !(NORM == KF_NORM_SOFTMAX && sizeof(T) == 2) && ((const void*)X != (const void*)Y || ldx == ldy) && M >= 2ll * sms &&
+        env_tpr == 0 && env_ring != 0) {
+        const size_t vecs = (NORM == KF_NORM_SOFTMAX ? 0 : (NORM == KF_NORM_LAYERNORM ? 2 : 1)) * grow_bytes;
+        const size_t budget = 226 * 1024 - 1024;             // reductions, flags and barriers fit the last KiB
+        const int total = budget > vecs ? (int)((budget - vecs) / grow_bytes) : 0;
+        int ng = 4;                                          // groups: as many as get two slots each
+        while (ng >= 1 && total < 2 * ng) ng >>= 1;
+        if (ng >= 1) {
+            int slots = total - total % ng;
+            if (slots > 3 * ng) slots = 3 * ng;
+            const size_t smem = (size_t)slots * grow_bytes + vecs + 512 + 32 + 2 * (size_t)slots * 8;
+            const int grid = (int)(M < sms ? M : sms);
+            switch (ng) {
+            case 4: return launch_gring<T, NORM, 4>(x, ldx, y, ldy, M, N, slots, grid, smem, g, b, rn.eps, st);
+            case 2: return launch_gring<T, NORM, 8>(x, ldx, y, ldy, M, N, slots, grid, smem, g, b, rn.eps, st);
+            default: return launch_gring<T, NORM, 16>(x, ldx, y, ldy, M, N, slots, grid, smem, g, b, rn.eps, st);
+            }
         }
     }
     // threads per row / vectors per thread: one warp per row while a row fits 16 vectors a lane

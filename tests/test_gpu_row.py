@@ -64,6 +64,39 @@ def test_row_ops_ring_kernel(kf, dtype, M, N):
     kf.row_layernorm(big[:, :N], dg, db, 1e-5, out=out[:, :N])
     assert_parity(to_f64(out[:, :N]), kfo.row_layernorm(X, g, b, 1e-5), dtype, "ring ln padded")
     assert bool((out[:, N:] == 5.0).all())
+    # in place (exact alias): a row is stored after its own copy has landed
+    kf.row_layernorm(big[:, :N], dg, db, 1e-5, out=big[:, :N])
+    assert_parity(to_f64(big[:, :N]), kfo.row_layernorm(X, g, b, 1e-5), dtype, "ring ln in place")
+    assert bool((big[:, N:] == 3.0).all())
+    soft = dX.clone()
+    kf.row_softmax(soft, out=soft)
+    assert_parity(to_f64(soft), kfo.row_softmax(X), dtype, "ring softmax in place")
+
+
+# rows beyond one warp's reach with enough of them for persistent CTAs: a slot per row, shared by a group of
+# 4, 8 or 16 warps (row bytes 16 Ki, 32 Ki, 64 Ki and ragged lengths between), out of place and in place
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("M,N", [(700, 8192), (333, 16384), (301, 32768), (450, 4104), (320, 12296), (310, 24584)])
+def test_row_ops_group_ring_kernel(kf, dtype, M, N):
+    if dtype == "f32":
+        N //= 2                                     # same row bytes in both types
+    X, g, b = _draw(300 + N, M, N, dtype, std=1.5, shift=0.75)
+    dX, dg, db = to_device(X, dtype), to_device(g, dtype), to_device(b, dtype)
+    ref_ln, ref_sm, ref_rms = kfo.row_layernorm(X, g, b, 1e-5), kfo.row_softmax(X), kfo.row_rmsnorm(X, g, 1e-6)
+    assert_parity(to_f64(kf.row_layernorm(dX, dg, db, 1e-5)), ref_ln, dtype, f"group ring ln {M}x{N}")
+    assert_parity(to_f64(kf.row_softmax(dX)), ref_sm, dtype, f"group ring softmax {M}x{N}")
+    assert_parity(to_f64(kf.row_rmsnorm(dX, dg, 1e-6)), ref_rms, dtype, f"group ring rms {M}x{N}")
+    assert_parity(to_f64(kf.row_layernorm(dX, None, None, 1e-5)), kfo.row_layernorm(X, None, None, 1e-5), dtype, "group ring ln plain")
+    # in place, on a padded pitch, canary columns untouched
+    big = torch.full((M, N + 16), 3.0, dtype=dX.dtype, device="cuda")
+    big[:, :N] = dX
+    kf.row_softmax(big[:, :N], out=big[:, :N])
+    assert_parity(to_f64(big[:, :N]), ref_sm, dtype, "group ring softmax in place")
+    assert bool((big[:, N:] == 3.0).all())
+    big[:, :N] = dX
+    kf.row_layernorm(big[:, :N], dg, db, 1e-5, out=big[:, :N])
+    assert_parity(to_f64(big[:, :N]), ref_ln, dtype, "group ring ln in place")
+    kf.check_device_status()
 
 
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
