@@ -1,4 +1,4 @@
-// Small fp32 linear + epilogue + row-norm calls (M <= 256, N <= 512, below the tensor-core gate): latency decides
+// Small fp32 linear + epilogue + row-norm calls (M <= 512, N <= 512, below the tensor-core gate): latency decides
 // them, not throughput, so the work of a row is spread over a thread-block cluster instead of held in one CTA.
 //
 //   cluster of 8 CTAs = 8 rows x all N columns; CTA r owns columns [r NC, (r+1) NC), NC = ceil(N / 8)
@@ -26,7 +26,7 @@ constexpr int kRowsCl = 8;           // rows per cluster, one warp each after th
 constexpr int kThreadsCl = 256;
 
 template <int CPL>                   // columns per lane: 1 (NC <= 32) or 2 (NC <= 64)
-__global__ void __launch_bounds__(kThreadsCl)
+__global__ void __launch_bounds__(kThreadsCl, 2)     // two CTAs per SM: a GPC then holds two clusters per 8 SMs
 simt_cluster_kernel(const float* __restrict__ X, long long ldx, const float* __restrict__ W, long long ldw, float* Y,
                     long long ldy, int M, int N, int K, const float* __restrict__ bias, const float* res,
                     long long ldr, int act, float scale, int norm, const float* __restrict__ gamma,
@@ -45,7 +45,7 @@ simt_cluster_kernel(const float* __restrict__ X, long long ldx, const float* __r
 
     cg::cluster_group cluster = cg::this_cluster();
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
-    const int rank = (int)cluster.block_rank();
+    const int rank = (int)(blockIdx.x % kCl);                // = the CTA's rank in its cluster (1-D clusters of kCl)
     const int m0 = (int)(blockIdx.x / kCl) * kRowsCl;
     const int NC = (N + kCl - 1) / kCl;
     const int n_base = rank * NC;
@@ -235,7 +235,7 @@ cudaError_t launch_cluster(const float* X, long long ldx, const float* W, long l
     at[0].val.clusterDim.y = 1;
     at[0].val.clusterDim.z = 1;
     lc.attrs = at;
-    lc.numAttrs = 1;
+    lc.numAttrs = rn.norm != KF_NORM_NONE ? 1 : 0;           // without a row-norm nothing crosses CTAs: a plain grid
     return cudaLaunchKernelEx(&lc, simt_cluster_kernel<CPL>, X, ldx, W, ldw, Y, ldy, (int)M, (int)N, (int)K,
                               static_cast<const float*>(ep.bias), static_cast<const float*>(ep.residual), ep.ldr,
                               ep.act, ep.scale, rn.norm, static_cast<const float*>(rn.gamma),
@@ -246,12 +246,14 @@ cudaError_t launch_cluster(const float* X, long long ldx, const float* W, long l
 
 // fp32 with 16-byte aligned rows (the caller checks pointers and pitches) and K a multiple of 4; rows of 64 to
 // 512 columns (shorter ones would leave most lanes of a CTA without a column).  Only where latency decides:
-// at most 256 rows (32 clusters, two CTAs per SM) -- with many clusters resident the cluster barriers wait on
-// time-sliced neighbours and the row-resident kernel wins (2048 x 512 x 28 with softmax: 82 us here, 27 there;
-// 256 x 128 x 512: 22 here, 33 there; 64 x 512 x 900: 20 here, 104 there) -- and a W of at least 64 KiB,
-// below which the row-resident kernel's single CTA per row reads it as quickly (16 x 64 x 16: 8 us there, 10 here)
+// at most 512 rows (64 clusters) -- a cluster of 8 needs 8 SMs of one GPC at the same time, so a B200 holds
+// two clusters per GPC and CTA slot (the kernel is kept to 128 registers for two CTAs per SM: with one, C1's
+// 16 clusters ran in two waves, 14.3 us instead of 10.2), and further clusters wait for whole clusters to
+// leave (1024 x 256 x 112 with softmax: 29 us here, 16 for the row-resident kernel; 512 x 512 x 112: 16 here,
+// 22 there; 64 x 512 x 900: 20 here, 104 there) -- and a W of at least 64 KiB, below which the row-resident
+// kernel's single CTA per row reads it as quickly (16 x 64 x 16: 8 us either way)
 bool simt_cluster_ok(long long M, long long N, long long K) {
-    return N >= 64 && N <= kCl * 64 && K % 4 == 0 && M <= 256 && N * K >= 16384;
+    return N >= 64 && N <= kCl * 64 && K % 4 == 0 && M <= 512 && N * K >= 16384;
 }
 
 cudaError_t launch_simt_cluster(const void* X, long long ldx, const void* W, long long ldw, void* Y, long long ldy,

@@ -77,7 +77,8 @@ def test_fp32_rownorm_row_resident(kf, norm, M, N, K):
                                    (100, 200, 260),      # 25 columns per CTA, a second slab of 4
                                    (9, 264, 516),        # 33 columns per CTA: two per lane, five slabs of 128
                                    (77, 68, 1028),       # 9 columns per CTA, the last CTA has 5
-                                   (256, 512, 32)])      # the most rows and the longest row this kernel takes
+                                   (256, 512, 32),       # the longest row this kernel takes
+                                   (509, 256, 64)])      # 64 clusters, the last with 5 rows
 def test_fp32_small_calls_rows_over_a_cluster(kf, norm, M, N, K):
     """Small aligned fp32 calls: 8 rows per cluster of 8 CTAs, each CTA an eighth of the columns, the row
     statistics merged through distributed shared memory."""
