@@ -31,6 +31,7 @@ def candidates(config: str):
         return
     if config == "c1":
         yield {}, "table default"
+        yield {"KF_TILE_OVERRIDE": "kernel=1"}, "row-resident CUDA-core kernel (one CTA per row)"
         yield {"KF_TILE_OVERRIDE": "kernel=2"}, "tiled CUDA-core kernel + row kernel"
         return
     for cg in (2, 1):               # cg=1 on more than one row block runs the generic form of the kernel
@@ -53,7 +54,9 @@ def descriptors(config: str, label: str):
     if config == "c2":
         return (3, 1, 2) if label.startswith("ring") else (1, 1, 2)
     if config == "c1":
-        return (2, 1, 1) if label.startswith("table") else (2, 0, 1)
+        if label.startswith("table"):
+            return (2, 1, 3)        # rows over clusters: statistics cross CTAs (distributed shared memory)
+        return (2, 1, 1) if label.startswith("row-resident") else (2, 0, 1)
     if config == "c3":
         return (3, 1, 1)
     return (3, 2, 3)
