@@ -241,6 +241,87 @@ simt_tiled_kernel(const T* __restrict__ X, long long ldx, const T* __restrict__ 
     }
 }
 
+// ------------------------------------------------------------------------------ tiled 128x128x16
+// The same contract as the 64x64 kernel for problems with enough 128 x 128 tiles to fill the device: 8 x 8
+// outputs per thread (two groups of 4 rows and of 4 columns, 64 apart, so that the 16-byte shared-memory
+// reads of a quarter-warp are contiguous), and the next k-slab on its way from global memory into
+// registers while the current one is multiplied out of shared memory.
+constexpr int kBM2 = 128, kBN2 = 128, kBK2 = 16;
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads, 2)
+simt_tiled128_kernel(const T* __restrict__ X, long long ldx, const T* __restrict__ W, long long ldw, T* Y,
+                     long long ldy, long long M, long long N, long long K, const T* __restrict__ bias, const T* res,
+                     long long ldr, int act, float scale) {
+    __shared__ __align__(16) float As[2][kBK2][kBM2];
+    __shared__ __align__(16) float Bs[2][kBK2][kBN2];
+    const int t = threadIdx.x;
+    const int tx = t % 16, ty = t / 16;
+    const long long m0 = (long long)blockIdx.y * kBM2, n0 = (long long)blockIdx.x * kBN2;
+    const int lrow = t / 2, lk = (t % 2) * 8;           // loader: 128 rows x 16 k, 8 consecutive k per thread
+    const bool a_ok = m0 + lrow < M, b_ok = n0 + lrow < N;
+    const T* xa = X + (m0 + lrow) * ldx;
+    const T* wb = W + (n0 + lrow) * ldw;
+
+    float acc[8][8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
+
+    float ra[8], rb[8];
+    auto fetch = [&](long long k0) {
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const long long k = k0 + lk + q;
+            ra[q] = (a_ok && k < K) ? Elem<T>::load(xa + k) : 0.f;
+            rb[q] = (b_ok && k < K) ? Elem<T>::load(wb + k) : 0.f;
+        }
+    };
+    auto stash = [&](int buf) {
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            As[buf][lk + q][lrow] = ra[q];
+            Bs[buf][lk + q][lrow] = rb[q];
+        }
+    };
+    if (K > 0) {
+        fetch(0);
+        stash(0);
+    }
+    __syncthreads();
+    int buf = 0;
+    for (long long k0 = 0; k0 < K; k0 += kBK2, buf ^= 1) {
+        const bool more = k0 + kBK2 < K;
+        if (more) fetch(k0 + kBK2);                      // in flight during the arithmetic below
+#pragma unroll
+        for (int kk = 0; kk < kBK2; ++kk) {
+            const float4 a0 = *reinterpret_cast<const float4*>(&As[buf][kk][ty * 4]);
+            const float4 a1 = *reinterpret_cast<const float4*>(&As[buf][kk][64 + ty * 4]);
+            const float4 b0 = *reinterpret_cast<const float4*>(&Bs[buf][kk][tx * 4]);
+            const float4 b1 = *reinterpret_cast<const float4*>(&Bs[buf][kk][64 + tx * 4]);
+            const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+            const float bv[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+#pragma unroll
+                for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+        }
+        if (more) stash(buf ^ 1);                        // the other buffer was last read before the previous barrier
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const long long m = m0 + (i < 4 ? ty * 4 + i : 64 + ty * 4 + (i - 4));
+        if (m >= M) continue;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const long long n = n0 + (j < 4 ? tx * 4 + j : 64 + tx * 4 + (j - 4));
+            if (n < N) Elem<T>::store(Y + m * ldy + n, epilogue_elem<T>(acc[i][j], m, n, bias, res, ldr, act, scale));
+        }
+    }
+}
+
 template <typename T, int BM, int NPT>
 cudaError_t launch_rows(const T* X, long long ldx, const T* W, long long ldw, T* Y, long long ldy, long long M,
                         long long N, long long K, const EpilogueParams& ep, const RowNormParams& rn,
@@ -283,12 +364,22 @@ cudaError_t launch_typed(const void* Xv, long long ldx, const void* Wv, long lon
         if (N <= 1024) return launch_rows_bm<T, 4>(X, ldx, W, ldw, Y, ldy, M, N, K, ep, rn, st, grid_out);
         return launch_rows_bm<T, 8>(X, ldx, W, ldw, Y, ldy, M, N, K, ep, rn, st, grid_out);
     }
-    const long long gx = (N + kTN - 1) / kTN, gy = (M + kTM - 1) / kTM;
-    if (gx > 0x7FFFFFFFll || gy > 65535) return cudaErrorInvalidConfiguration;
-    if (grid_out) *grid_out = (int)(gx * gy);
-    simt_tiled_kernel<T><<<dim3((unsigned)gx, (unsigned)gy), kThreads, 0, st>>>(
-        X, ldx, W, ldw, Y, ldy, M, N, K, static_cast<const T*>(ep.bias), static_cast<const T*>(ep.residual),
-        ep.ldr, ep.act, ep.scale);
+    // 128 x 128 tiles once there are a few dozen of them (8 x 8 outputs per thread: a quarter of the
+    // shared-memory traffic per multiply-add, and the next slab prefetched), else 64 x 64
+    const long long gx2 = (N + kBN2 - 1) / kBN2, gy2 = (M + kBM2 - 1) / kBM2;
+    if (gx2 * gy2 >= 24 && gy2 <= 65535 && gx2 <= 0x7FFFFFFFll) {
+        if (grid_out) *grid_out = (int)(gx2 * gy2);
+        simt_tiled128_kernel<T><<<dim3((unsigned)gx2, (unsigned)gy2), kThreads, 0, st>>>(
+            X, ldx, W, ldw, Y, ldy, M, N, K, static_cast<const T*>(ep.bias), static_cast<const T*>(ep.residual),
+            ep.ldr, ep.act, ep.scale);
+    } else {
+        const long long gx = (N + kTN - 1) / kTN, gy = (M + kTM - 1) / kTM;
+        if (gx > 0x7FFFFFFFll || gy > 65535) return cudaErrorInvalidConfiguration;
+        if (grid_out) *grid_out = (int)(gx * gy);
+        simt_tiled_kernel<T><<<dim3((unsigned)gx, (unsigned)gy), kThreads, 0, st>>>(
+            X, ldx, W, ldw, Y, ldy, M, N, K, static_cast<const T*>(ep.bias), static_cast<const T*>(ep.residual),
+            ep.ldr, ep.act, ep.scale);
+    }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess || rn.norm == KF_NORM_NONE) return e;
     return launch_row_norm(Yv, ldy, Yv, ldy, M, N, sizeof(T) == 4 ? KF_F32 : KF_BF16, rn, st);

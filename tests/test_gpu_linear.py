@@ -93,13 +93,26 @@ def test_fp32_small_calls_rows_over_a_cluster(kf, norm, M, N, K):
 
 @pytest.mark.parametrize("norm", ["none", "softmax", "layernorm"])
 def test_fp32_tiled_kernel_and_unfused_rownorm(kf, norm):
-    M, N, K = 130, 2500, 70                         # N > 2048: tiled GEMM, row op as a second in-place kernel
+    M, N, K = 130, 2300, 70                         # N > 2048: tiled GEMM, row op as a second in-place kernel
     p = make("f32", M, N, K, seed=13, act="silu", norm=norm, res=True, scale=0.5)
     assert kf.tile_config(M, N, K, torch.float32, norm)["kernel"] == 2
     assert_parity(run(kf, p), oracle_of(p), "f32", f"tiled {norm}")
     p = make("f32", 1500, 96, 33, seed=14, act="relu")           # tall: tiled kernel without a row op
     assert kf.tile_config(1500, 96, 33, torch.float32, "none")["kernel"] == 2
     assert_parity(run(kf, p), oracle_of(p), "f32", "tall")
+
+
+@pytest.mark.parametrize("dtype,M,N,K,norm", [("f32", 700, 2500, 70, "softmax"),      # 6 x 20 tiles of 128 x 128
+                                               ("f32", 1030, 1541, 131, "none"),     # ragged in M, N and K
+                                               ("bf16", 1030, 1541, 129, "none")])   # odd pitches: no TMA
+def test_large_tile_cuda_core_kernel(kf, dtype, M, N, K, norm):
+    """Calls the tensor-core paths cannot take (odd pitches, small fp32 work on long rows) with enough 128 x 128
+    tiles for every SM run the 8 x 8-per-thread kernel."""
+    p = make(dtype, M, N, K, seed=19 + K, act="gelu_tanh", norm=norm, res=True, scale=0.5)
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    cfg = kf.tile_config(M, N, K, tdt, norm, aligned=(N % 8 == 0 and K % 8 == 0))
+    assert (cfg["kernel"], cfg["bm"], cfg["bn"]) == (2, 128, 128)
+    assert_parity(run(kf, p), oracle_of(p), dtype, f"tiled128 {dtype} {M}x{N}x{K}")
 
 
 def test_bf16_unaligned_goes_to_cuda_cores(kf):
