@@ -21,8 +21,8 @@
 // Row-norm (split-N): a row of N outputs spans N/128 sub-tiles owned by different warps and CTAs.
 // With the sub-tile row in registers the thread gathers its statistics, then turns the values into
 // a 16-bit intermediate stored in Y -- softmax: bf16 exp(a - tile max); LayerNorm / RMSNorm: fp16
-// (a - tile shift) * 2^-e with a per-row, per-tile power-of-two block scale, so the intermediate
-// carries 11 significant bits relative to the largest deviation of the tile row.  The per-row
+// (a - tile shift) * 2^-e with a per-row, per-tile power-of-two block scale 2^e above sqrt(sum of squared
+// deviations), which keeps every value inside fp16's range with its 11 significant bits.  The per-row
 // partial {shift or max, sum, sum of squares, 2^e} goes to the workspace; the finishing kernel
 // merges the partials of a row (online-softmax rescaling / Chan's merge) and rescales in place.
 //
@@ -485,7 +485,7 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             // beyond N (ragged last chunk) are set to the neutral value of the statistic
             float st_shift = 0.f, st_s1 = 0.f, st_s2 = 0.f, st_scale = 1.f, mult = 1.f;
             float2 s1[2] = {f2(0.f), f2(0.f)}, s2[2] = {f2(0.f), f2(0.f)};
-            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY}, am[4] = {0.f, 0.f, 0.f, 0.f};
+            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
             for (int c = 0; c < kSub / 32; ++c) {
                 if (c < nchunks) {
@@ -525,8 +525,6 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
                         for (int i = 0; i < 16; ++i) {
                             s1[i & 1] = __fadd2_rn(s1[i & 1], a[i]);
                             s2[i & 1] = __ffma2_rn(a[i], a[i], s2[i & 1]);
-                            am[(2 * i) & 3] = fmaxf(am[(2 * i) & 3], fabsf(a[i].x));
-                            am[(2 * i + 1) & 3] = fmaxf(am[(2 * i + 1) & 3], fabsf(a[i].y));
                         }
                     }
 #pragma unroll
@@ -541,9 +539,12 @@ tc_linear_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             } else if (norm != KF_NORM_NONE) {
                 st_s1 = (s1[0].x + s1[0].y) + (s1[1].x + s1[1].y);
                 st_s2 = (s2[0].x + s2[0].y) + (s2[1].x + s2[1].y);
-                const float amax = fmaxf(fmaxf(am[0], am[1]), fmaxf(am[2], am[3]));
-                // power-of-two block scale: stored fp16 values lie in (-2, 2)
-                uint32_t eb = (__float_as_uint(amax) >> 23) & 0xFFu;
+                // power-of-two block scale from a bound on the largest deviation, sqrt(sum of squares) >= max |d|
+                // (no running maximum in the loop above): stored fp16 values lie in (-2, 2).  The bound may
+                // exceed the maximum by sqrt(128); fp16 being a floating-point format, that costs no
+                // significant bits, it only moves the values below 2^-14 of the scale into subnormals.
+                const float bound = sqrtf(st_s2);
+                uint32_t eb = ((__float_as_uint(bound) >> 23) & 0xFFu) + 1u;     // (+1: the square root may round down)
                 eb = min(max(eb, 1u), 253u);
                 st_scale = __uint_as_float(eb << 23);
                 mult = __uint_as_float((254u - eb) << 23);
