@@ -246,6 +246,20 @@ def test_tc_residual_may_alias_output(kf):
     assert_parity(to_f64(y), oracle_of(p), "bf16", "aliased residual")
 
 
+@pytest.mark.parametrize("M,N,K,norm", [(100, 256, 256, "layernorm"),     # rows over clusters
+                                         (100, 256, 256, "none"),          # the same kernel as a plain grid
+                                         (700, 2500, 70, "none"),          # 128 x 128 tiled kernel
+                                         (515, 1028, 132, "rmsnorm")])     # past the 3xTF32 gate: demoted, Y holds running sums there
+def test_fp32_residual_may_alias_output(kf, M, N, K, norm):
+    p = make("f32", M, N, K, seed=33 + N, act="gelu_tanh", norm=norm, res=True, scale=0.5)
+    d = problem_to_device(p)
+    out = d["residual"]
+    y = kf.linear_epilogue_rownorm(d["X"], d["W"], d["bias"], p.act, p.scale, out, p.norm, d["gamma"], d["beta"], p.eps, out=out)
+    kf.check_device_status()
+    assert y.data_ptr() == out.data_ptr()
+    assert_parity(to_f64(y), oracle_of(p), "f32", f"aliased residual {norm} {M}x{N}x{K}")
+
+
 def test_tc_padded_pitches_and_canaries(kf):
     """Row pitches larger than the rows; memory between rows and behind the output must stay untouched."""
     p = make("bf16", 150, 264, 136, seed=31, act="relu", norm="layernorm", res=True)
